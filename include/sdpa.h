@@ -1,0 +1,114 @@
+/*
+ * sdpa.h - C ABI of the B200 (sm_100a) bf16 scaled-dot-product-attention library.
+ *
+ * One forward and one backward entry point over packed (variable-length) batches with
+ * grouped-query heads.  Every step of the path runs in this library's own CUDA kernels
+ * (TMA-staged tiles, tcgen05 MMAs with TMEM accumulators); there is no CPU path and no call
+ * into any attention/GEMM library.
+ *
+ * Conventions shared by all entry points
+ * --------------------------------------
+ *  - All tensor pointers are DEVICE pointers, 16-byte aligned, contiguous, caller-owned.
+ *    The library never allocates or frees memory; calls are asynchronous on `stream`
+ *    (a cudaStream_t passed as void*, may be 0) and every buffer must stay alive until the
+ *    stream has passed the call.
+ *  - Token-major packed layout.  T = total_tokens = cu_seqlens[B].
+ *        q, o, dout, dq : bf16 [T, Hq,  D]
+ *        k, v, dk, dv   : bf16 [T, Hkv, D]
+ *        lse            : fp32 [Hq, T]
+ *        cu_seqlens     : int32 [B + 1] in device memory, cu_seqlens[0] = 0, non-decreasing;
+ *                         sequence b owns token rows cu_seqlens[b] .. cu_seqlens[b+1]-1 of every
+ *                         tensor (self-attention: queries and keys of a sequence have equal length).
+ *  - Grouped-query attention: query head h reads kv head h / (Hq / Hkv).
+ *  - causal != 0: query i of a sequence attends to keys 0..i of that sequence
+ *    (lower-triangular mask); causal == 0: to all keys of its sequence.
+ *  - Supported: D in {64, 128}; Hq a multiple of Hkv; scale finite and > 0; sequences of any
+ *    length >= 0 (empty sequences and T = 0 are valid no-ops).
+ *  - max_seqlen must be >= the longest sequence; total_tokens must equal cu_seqlens[B].  They
+ *    size the launch grid and the TMA tensor maps without a device-to-host read of cu_seqlens.
+ *    A cu_seqlens that contradicts them is reported through sdpa_query_status
+ *    (SDPA_STATUS_BAD_CU_SEQLENS); outputs are then unspecified but no out-of-bounds access happens.
+ *
+ * Return value of the launching calls: SDPA_OK (0) when the work was enqueued, a negative
+ * SDPA_ERR_* code when the call was rejected before any launch.  Problems found on the device
+ * (a bounded wait that ran out, inconsistent cu_seqlens) are latched in a per-device status word
+ * read by sdpa_query_status.
+ */
+#ifndef SDPA_B200_H_
+#define SDPA_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SDPA_OK 0
+#define SDPA_ERR_NULL (-1)      /* a required pointer is null */
+#define SDPA_ERR_ALIGN (-2)     /* a tensor pointer is not 16-byte aligned */
+#define SDPA_ERR_SHAPE (-3)     /* unsupported D, Hq % Hkv != 0, B < 1, negative sizes, bad scale */
+#define SDPA_ERR_WORKSPACE (-4) /* workspace missing, misaligned or too small */
+#define SDPA_ERR_ARCH (-5)      /* current device is not compute capability 10.x */
+#define SDPA_ERR_CUDA (-6)      /* a CUDA runtime/driver call failed; see sdpa_last_cuda_error */
+
+#define SDPA_STATUS_TIMEOUT 1        /* a device-side wait gave up; outputs of that call are invalid */
+#define SDPA_STATUS_BAD_CU_SEQLENS 2 /* cu_seqlens contradicts total_tokens / max_seqlen */
+#define SDPA_STATUS_INTERNAL 3       /* a kernel found its own launch preconditions violated */
+
+/*
+ * Forward pass (paper, appendix "Workloads": MHA forward, causal and non-causal, returns a bf16
+ * output and an fp32 log-sum-exp; "Generalization attention workloads": GQA over ragged batches;
+ * evaluation order: the online-softmax tile loop of the corrected Algorithm 2, whose epilogue
+ * defines O = diag(l)^-1 O and L = m + log l).
+ *   o[r,h,:]  = sum_j softmax_j(scale * q[r,h,:] . k[j,g,:]) v[j,g,:]   over the allowed keys j
+ *   lse[h,r]  = natural log of sum_j exp(scale * q[r,h,:] . k[j,g,:])   over the allowed keys j
+ * q, k, v are read; o (bf16, round to nearest even) and lse (fp32) are overwritten for every
+ * token row of every sequence.
+ */
+int sdpa_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+             const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D, int causal, float scale,
+             int total_tokens, int max_seqlen, void* stream);
+
+/*
+ * Bytes of scratch sdpa_bwd needs for these sizes (fp32 dQ accumulator [T,Hq,D] plus the fp32
+ * row terms D_i [Hq,T]); 0 on invalid arguments.  The workspace must be 256-byte aligned device
+ * memory; its contents on entry do not matter and are unspecified on exit.
+ */
+size_t sdpa_bwd_workspace_bytes(int B, int Hq, int Hkv, int D, int total_tokens, int max_seqlen);
+
+/*
+ * Backward pass (paper, appendix "Workloads": MHA backward consumes Q, K, V, the forward output,
+ * its upstream gradient and the log-sum-exp, and returns bf16 gradients of Q, K, V).  With P
+ * recomputed as exp(scale * q.k - lse):
+ *   D_i = dout_i . o_i      dP = dout V^T      dS = P * (dP - D_i)
+ *   dq = scale * dS K       dk = scale * dS^T Q       dv = P^T dout
+ * dk and dv are summed over the Hq / Hkv query heads that share a kv head.  o and lse must be the
+ * outputs of sdpa_fwd on the same q, k, v, cu_seqlens, causal and scale.  dq, dk, dv are
+ * overwritten (not accumulated into).  dq partial sums from different key tiles are combined
+ * with floating-point atomics, so dq may differ in the last bits from run to run.
+ */
+int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse,
+             const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B,
+             int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
+             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Waits for `stream`, then returns the current device's status word (0 = no device-side problem
+ * since the last query; otherwise an SDPA_STATUS_* code) and clears it.  *site (may be null)
+ * receives an internal identifier of the wait that gave up.  Returns SDPA_ERR_CUDA if the
+ * synchronisation or the copy failed.
+ */
+int sdpa_query_status(void* stream, int* site);
+
+/* Static, human-readable name of a return or status code. */
+const char* sdpa_status_string(int code);
+
+/* The cudaError_t (as int) of the most recent failed runtime call made by this library on the
+ * calling thread, or the CUresult of a failed tensor-map encode; 0 if none. */
+int sdpa_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDPA_B200_H_ */

@@ -1,0 +1,130 @@
+"""Python binding of the C ABI in include/sdpa.h: argument marshalling only.
+
+Every step of the attention path runs in the CUDA library; torch supplies device memory and
+streams.  There is no fallback: if the shared library is missing or cannot be loaded, or no
+CUDA device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsdpa_b200.so")
+_LIB = None
+
+SDPA_OK = 0
+EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
+           "sdpa_status_string", "sdpa_last_cuda_error")
+
+
+class SdpaError(RuntimeError):
+    pass
+
+
+def load():
+    """Load libsdpa_b200.so (built by paper_2608_17379_b200.build) and declare its signatures."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    if not os.path.exists(LIB_PATH):
+        raise SdpaError(f"{LIB_PATH} is missing: run `python -m paper_2608_17379_b200.build` "
+                        "(there is no CPU or library fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    lib.sdpa_fwd.restype = ci
+    lib.sdpa_fwd.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, ci, vp]
+    lib.sdpa_bwd_workspace_bytes.restype = ctypes.c_size_t
+    lib.sdpa_bwd_workspace_bytes.argtypes = [ci] * 6
+    lib.sdpa_bwd.restype = ci
+    lib.sdpa_bwd.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp, ctypes.c_size_t, vp]
+    lib.sdpa_query_status.restype = ci
+    lib.sdpa_query_status.argtypes = [vp, ctypes.POINTER(ci)]
+    lib.sdpa_status_string.restype = ctypes.c_char_p
+    lib.sdpa_status_string.argtypes = [ci]
+    lib.sdpa_last_cuda_error.restype = ci
+    lib.sdpa_last_cuda_error.argtypes = []
+    _LIB = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load().sdpa_status_string(int(code)).decode()
+
+
+def _check(rc: int, what: str):
+    if rc != SDPA_OK:
+        lib = load()
+        raise SdpaError(f"{what} failed: {rc} ({status_string(rc)}), cuda error {lib.sdpa_last_cuda_error()}")
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _dims(q, k):
+    assert q.dtype == torch.bfloat16 and k.dtype == torch.bfloat16
+    assert q.is_contiguous() and k.is_contiguous() and q.dim() == 3 and k.dim() == 3
+    T, Hq, D = q.shape
+    return T, Hq, k.shape[1], D
+
+
+def sdpa_fwd(q, k, v, cu_seqlens, max_seqlen: int, causal: bool, scale: float, o=None, lse=None, stream=None):
+    """q [T,Hq,D], k,v [T,Hkv,D] bf16 CUDA tensors, cu_seqlens int32 [B+1] on the device.
+
+    Returns (o bf16 [T,Hq,D], lse fp32 [Hq,T]); asynchronous on ``stream`` (default: current)."""
+    lib = load()
+    T, Hq, Hkv, D = _dims(q, k)
+    B = cu_seqlens.numel() - 1
+    assert cu_seqlens.dtype == torch.int32 and cu_seqlens.is_cuda
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((Hq, T), dtype=torch.float32, device=q.device)
+    rc = lib.sdpa_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(cu_seqlens), B, Hq, Hkv, D,
+                      int(bool(causal)), float(scale), T, int(max_seqlen), _stream_ptr(stream))
+    _check(rc, "sdpa_fwd")
+    return o, lse
+
+
+def sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen) -> int:
+    return int(load().sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen))
+
+
+def sdpa_bwd(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, scale: float,
+             dq=None, dk=None, dv=None, workspace=None, stream=None):
+    """Gradients (dq, dk, dv) bf16 of sum(dout * O); o and lse are the outputs of sdpa_fwd."""
+    lib = load()
+    T, Hq, Hkv, D = _dims(q, k)
+    B = cu_seqlens.numel() - 1
+    need = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, T, int(max_seqlen))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk is None:
+        dk = torch.empty_like(k)
+    if dv is None:
+        dv = torch.empty_like(v)
+    rc = lib.sdpa_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
+                      _ptr(cu_seqlens), B, Hq, Hkv, D, int(bool(causal)), float(scale), T, int(max_seqlen),
+                      _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
+    _check(rc, "sdpa_bwd")
+    return dq, dk, dv
+
+
+def query_status(stream=None):
+    """Synchronise the stream and return (status, site) of the device status word (0 = fine)."""
+    site = ctypes.c_int(0)
+    rc = load().sdpa_query_status(_stream_ptr(stream), ctypes.byref(site))
+    if rc < 0:
+        _check(rc, "sdpa_query_status")
+    return rc, site.value

@@ -1,0 +1,357 @@
+// Forward attention kernel for sm_100a.
+//
+// One CTA owns two consecutive 128-row query tiles of one (sequence, query head) and walks the
+// 128-row key/value tiles of that sequence.  Roles (warp-specialised, 12 warps):
+//   warps 0-3   softmax group of query tile 0 (thread = one query row)
+//   warps 4-7   softmax group of query tile 1
+//   warp  8     MMA issuer (one elected lane): S = Q K^T and O += P V with tcgen05.mma
+//   warp  9     TMA producer (one elected lane): Q tiles once, K/V tiles through an mbarrier ring
+//   warps 10-11 idle (they complete the third warpgroup so registers can be re-balanced)
+// TMEM (512 columns): S of tile 0 [0,128), S of tile 1 [128,256), O of tile 0 [256,256+D),
+// O of tile 1 [384,384+D).  bf16 P overwrites the first 64 columns of its S and feeds the second
+// MMA straight from TMEM.  While one group runs its softmax the tensor core works for the other.
+//
+// The loop is the online-softmax recurrence (running max m, running sum l, rescale of O when the
+// max moves); O is only rescaled when the max grew by more than 2^8 in the exp2 domain, otherwise
+// the stale max stays the reference, which changes nothing in exact arithmetic.
+#pragma once
+#include "ptx.cuh"
+
+namespace sdpa {
+
+struct FwdParams {
+    const int32_t* cu_seqlens;
+    __nv_bfloat16* o;
+    float* lse;
+    int* status;
+    int B, Hq, Hkv, T;
+    int causal;
+    int max_seqlen;
+    float scale;       // softmax scale
+    float scale_log2;  // scale * log2(e)
+};
+
+template <int D>
+struct FwdCfg {
+    static constexpr int kThreads = 384;
+    static constexpr int kTile = 128;
+    static constexpr int kTileBytes = kTile * D * 2;             // one Q, K or V tile
+    static constexpr int kAtomBytes = kTile * 128;               // one 64-column swizzle atom of a tile
+    static constexpr int kStages = (D == 128) ? 4 : 8;           // K/V ring slots
+    static constexpr int kSmemQ = 2 * kTileBytes;
+    static constexpr int kSmemRing = kStages * kTileBytes;
+    static constexpr int kSmemBars = 1024;
+    static constexpr int kSmemBytes = kSmemQ + kSmemRing + kSmemBars + 1024;  // + alignment slack
+    static constexpr int kKSteps = D / 16;                       // k-steps of S = Q K^T
+};
+
+enum FwdSite {
+    kSiteQFull = 1, kSiteKvFull = 2, kSiteKvEmpty = 3, kSiteSFull = 4, kSitePFull = 5, kSiteOFull = 6,
+    kSiteDrain = 7
+};
+
+template <int D>
+__global__ void __launch_bounds__(384, 1)
+sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
+    using Cfg = FwdCfg<D>;
+    constexpr int S = Cfg::kStages;
+
+    const int bh = blockIdx.x;
+    const int b = bh / p.Hq, h = bh % p.Hq;
+    const int g = h / (p.Hq / p.Hkv);
+    const int pair = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest (latest) query tiles first
+    const int r0 = p.cu_seqlens[b];
+    const int r1 = p.cu_seqlens[b + 1];
+    int L = r1 - r0;
+    if (L < 0 || r0 < 0 || r1 > p.T || L > p.max_seqlen) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
+        return;
+    }
+    const int q_start = pair * 256;
+    if (q_start >= L) return;
+
+    int n_kv[2];
+    const int n_kv_all = (L + 127) >> 7;
+    {
+        const bool has1 = (q_start + 128) < L;
+        n_kv[0] = p.causal ? (q_start >> 7) + 1 : n_kv_all;
+        n_kv[1] = has1 ? (p.causal ? ((q_start + 128) >> 7) + 1 : n_kv_all) : 0;
+    }
+    const int n_iter = max(n_kv[0], n_kv[1]);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;
+    uint8_t* sRing = smem + Cfg::kSmemQ;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kSmemQ + Cfg::kSmemRing);
+    uint64_t* q_full = bars;               // [2]
+    uint64_t* kv_full = bars + 2;          // [S]
+    uint64_t* kv_empty = bars + 2 + S;     // [S]
+    uint64_t* s_full = bars + 2 + 2 * S;   // [2]
+    uint64_t* p_full = s_full + 2;         // [2]
+    uint64_t* o_full = p_full + 2;         // [2]
+    uint64_t* drain = o_full + 2;          // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const WaitCtl ctl{p.status, abort_flag};
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&q_full[i], 1);
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_full[i], 128);
+            mbar_init(&o_full[i], 1);
+        }
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&kv_full[i], 1);
+            mbar_init(&kv_empty[i], 1);
+        }
+        mbar_init(drain, 1);
+        fence_mbar_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    if (warp == 9 && elect_one()) {
+        prefetch_tmap(&map_q);
+        prefetch_tmap(&map_k);
+        prefetch_tmap(&map_v);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp < 8) {
+        // ------------------------------------------------------------ softmax groups
+        setmaxnreg_inc<208>();
+        const int t = warp >> 2;                 // which query tile
+        const int row_in_tile = tid & 127;
+        const int row = q_start + t * 128 + row_in_tile;  // row inside the sequence
+        const bool valid = row < L;
+        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_base + t * 128;
+        const uint32_t tO = tmem + lane_base + 256 + t * 128;
+        float m = -INFINITY, l = 0.f;
+        const int n = n_kv[t];
+        bool ok = true;
+        for (int j = 0; j < n && ok; ++j) {
+            ok = mbar_wait_warp(&s_full[t], j & 1, ctl, kSiteSFull);
+            if (!ok) break;
+            tc_fence_after();
+            float s[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld_x32(tS + c * 32, r);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
+            }
+            tmem_wait_ld();
+            const int key0 = j * 128;
+            const bool diag = p.causal && (key0 + 127 > q_start + t * 128);
+            if (diag || key0 + 128 > L) {
+                const int lim = p.causal ? min(row, L - 1) : (L - 1);  // last allowed key
+#pragma unroll
+                for (int c = 0; c < 128; ++c)
+                    if (key0 + c > lim) s[c] = -INFINITY;
+            }
+            float mx = s[0];
+#pragma unroll
+            for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+            if (j == 0) {
+                m = mx;
+            } else {
+                const bool grow = (mx - m) * p.scale_log2 > 8.0f;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float m_new = fmaxf(m, mx);
+                    const float alpha = fast_exp2((m - m_new) * p.scale_log2);
+                    m = m_new;
+                    l *= alpha;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_x32(tO + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st_x32(tO + c * 32, r);
+                    }
+                }
+            }
+            const float neg_m = -m * p.scale_log2;
+            float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t r[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float e0 = fast_exp2(fmaf(s[c * 64 + 2 * i], p.scale_log2, neg_m));
+                    const float e1 = fast_exp2(fmaf(s[c * 64 + 2 * i + 1], p.scale_log2, neg_m));
+                    sum0 += e0;
+                    sum1 += e1;
+                    r[i] = pack_bf16x2(e0, e1);
+                }
+                tmem_st_x32(tS + c * 32, r);
+            }
+            l += sum0 + sum1;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&p_full[t]);
+        }
+        if (ok && n > 0) ok = mbar_wait_warp(&o_full[t], 0, ctl, kSiteOFull);
+        if (ok && n > 0) {
+            tc_fence_after();
+            const float inv_l = 1.0f / l;
+            __nv_bfloat16* orow = p.o + (static_cast<size_t>(r0 + row) * p.Hq + h) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_x32(tO + c * 32, r);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(r[8 * i + 0]) * inv_l, __uint_as_float(r[8 * i + 1]) * inv_l);
+                        w.y = pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv_l, __uint_as_float(r[8 * i + 3]) * inv_l);
+                        w.z = pack_bf16x2(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
+                        w.w = pack_bf16x2(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
+                    }
+                }
+            }
+            if (valid) p.lse[static_cast<size_t>(h) * p.T + r0 + row] = m * p.scale + logf(l);
+        }
+    } else {
+        setmaxnreg_dec<40>();
+        if (warp == 9) {
+            // -------------------------------------------------------- TMA producer
+            if (elect_one()) {
+                int it = 0;
+                auto load_tile = [&](const CUtensorMap* map, uint8_t* dst, uint64_t* bar, int head, int tok) {
+                    mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
+#pragma unroll
+                    for (int a = 0; a < D / 64; ++a) tma_load_3d(dst + a * Cfg::kAtomBytes, map, bar, a * 64, head, tok);
+                };
+                bool ok = true;
+                load_tile(&map_q, sQ, &q_full[0], h, r0 + q_start);
+                for (int j = 0; j < n_iter && ok; ++j) {
+                    for (int kv = 0; kv < 2 && ok; ++kv, ++it) {
+                        const int st = it % S;
+                        ok = mbar_wait(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
+                        if (!ok) break;
+                        load_tile(kv == 0 ? &map_k : &map_v, sRing + st * Cfg::kTileBytes, &kv_full[st], g,
+                                  r0 + j * 128);
+                        if (j == 0 && kv == 0 && n_kv[1] > 0)
+                            load_tile(&map_q, sQ + Cfg::kTileBytes, &q_full[1], h, r0 + q_start + 128);
+                    }
+                }
+                if (!ok) {
+                    // abandon: let the copies already issued land before the CTA exits
+                    for (int back = 1; back <= S && back <= it; ++back) {
+                        const int i2 = it - back;
+                        mbar_wait(&kv_full[i2 % S], (i2 / S) & 1, ctl, kSiteDrain);
+                    }
+                }
+            }
+        } else if (warp == 8) {
+            // -------------------------------------------------------- MMA issuer
+            if (elect_one()) {
+                constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
+                constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, false, true);
+                const uint32_t q_addr = smem_u32(sQ);
+                const uint32_t ring_addr = smem_u32(sRing);
+                auto issue_qk = [&](int t, int st) {
+                    const uint32_t a0 = q_addr + t * Cfg::kTileBytes;
+                    const uint32_t b0 = ring_addr + st * Cfg::kTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < Cfg::kKSteps; ++kk) {
+                        const uint32_t off = (kk >> 2) * Cfg::kAtomBytes + (kk & 3) * 32;
+                        umma_ss(tmem + t * 128, smem_desc_sw128(a0 + off, 0, 1024), smem_desc_sw128(b0 + off, 0, 1024),
+                                idesc_qk, kk > 0);
+                    }
+                };
+                auto issue_pv = [&](int t, int st, bool accumulate) {
+                    const uint32_t b0 = ring_addr + st * Cfg::kTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        umma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
+                                smem_desc_sw128(b0 + kk * 2048, Cfg::kAtomBytes, 1024), idesc_pv,
+                                (accumulate || kk > 0) ? 1u : 0u);
+                    }
+                };
+                bool ok = true;
+                int it = 0;  // ring consumer counter: K_j is item 2j, V_j is item 2j+1
+                ok = mbar_wait(&q_full[0], 0, ctl, kSiteQFull);
+                if (ok) ok = mbar_wait(&kv_full[0], 0, ctl, kSiteKvFull);
+                if (ok) {
+                    tc_fence_after();
+                    issue_qk(0, 0);
+                    umma_commit(&s_full[0]);
+                    if (n_kv[1] > 0) {
+                        ok = mbar_wait(&q_full[1], 0, ctl, kSiteQFull);
+                        if (ok) {
+                            tc_fence_after();
+                            issue_qk(1, 0);
+                            umma_commit(&s_full[1]);
+                        }
+                    }
+                    umma_commit(&kv_empty[0]);
+                    it = 1;
+                }
+                for (int j = 0; j < n_iter && ok; ++j) {
+                    const int st_v = it % S;
+                    ok = mbar_wait(&kv_full[st_v], (it / S) & 1, ctl, kSiteKvFull);
+                    if (!ok) break;
+                    ++it;
+                    const bool have_next = (j + 1) < n_iter;
+                    const int st_k = it % S;
+                    bool next_ready = false;
+                    for (int t = 0; t < 2 && ok; ++t) {
+                        if (j >= n_kv[t]) continue;
+                        ok = mbar_wait(&p_full[t], j & 1, ctl, kSitePFull);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(t, st_v, j > 0);
+                        if (j + 1 < n_kv[t]) {
+                            if (!next_ready) {
+                                ok = mbar_wait(&kv_full[st_k], (it / S) & 1, ctl, kSiteKvFull);
+                                if (!ok) break;
+                                tc_fence_after();
+                                next_ready = true;
+                            }
+                            issue_qk(t, st_k);
+                            umma_commit(&s_full[t]);
+                        } else {
+                            umma_commit(&o_full[t]);
+                        }
+                    }
+                    if (!ok) break;
+                    umma_commit(&kv_empty[st_v]);
+                    if (have_next) {
+                        umma_commit(&kv_empty[st_k]);
+                        ++it;
+                    }
+                }
+                if (!ok) {
+                    // abandon: wait (bounded) until the MMAs already issued have left the pipe
+                    umma_commit(drain);
+                    mbar_wait(drain, 0, ctl, kSiteDrain);
+                }
+            }
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace sdpa

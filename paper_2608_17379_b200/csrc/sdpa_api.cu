@@ -1,0 +1,275 @@
+// Host side of the C ABI declared in include/sdpa.h: argument checks, TMA tensor maps, launches.
+// Links against the CUDA runtime only; cuTensorMapEncodeTiled is fetched through
+// cudaGetDriverEntryPoint.  Nothing here allocates or frees device memory.
+#include "../../include/sdpa.h"
+
+#include <math.h>
+#include <mutex>
+
+#include "bwd_kernel.cuh"
+#include "fwd_kernel.cuh"
+
+namespace sdpa {
+
+__device__ int g_status_word;  // per-device status (0 = ok), latched by the kernels
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static thread_local int tl_last_cuda_error = 0;
+
+#define SDPA_CUDA_TRY(expr)                          \
+    do {                                             \
+        cudaError_t e__ = (expr);                    \
+        if (e__ != cudaSuccess) {                    \
+            tl_last_cuda_error = static_cast<int>(e__); \
+            (void)cudaGetLastError();                \
+            return SDPA_ERR_CUDA;                    \
+        }                                            \
+    } while (0)
+
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+    bool ready = false;
+    bool arch_ok = false;
+    int* status_ptr = nullptr;
+    int num_sms = 0;
+};
+static DeviceState g_dev[kMaxDevices];
+static std::mutex g_mutex;
+static EncodeTiledFn g_encode = nullptr;
+
+// Per-device one-time set-up: architecture check, status-word address, shared-memory opt-in.
+static int device_state(DeviceState** out) {
+    int dev = -1;
+    SDPA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SDPA_ERR_ARCH;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& st = g_dev[dev];
+    if (!st.ready) {
+        int major = 0;
+        SDPA_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        SDPA_CUDA_TRY(cudaDeviceGetAttribute(&st.num_sms, cudaDevAttrMultiProcessorCount, dev));
+        st.arch_ok = (major == 10);
+        if (st.arch_ok) {
+            if (!g_encode) {
+                void* fn = nullptr;
+                cudaDriverEntryPointQueryResult q;
+                SDPA_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+                if (fn == nullptr || q != cudaDriverEntryPointSuccess) {
+                    tl_last_cuda_error = static_cast<int>(cudaErrorNotSupported);
+                    return SDPA_ERR_CUDA;
+                }
+                g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+            }
+            void* sym = nullptr;
+            SDPA_CUDA_TRY(cudaGetSymbolAddress(&sym, g_status_word));
+            st.status_ptr = static_cast<int*>(sym);
+            SDPA_CUDA_TRY(cudaMemset(st.status_ptr, 0, sizeof(int)));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               FwdCfg<128>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               FwdCfg<64>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               BwdCfg<128>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               BwdCfg<64>::kSmemBytes));
+        }
+        st.ready = true;
+    }
+    *out = &st;
+    return st.arch_ok ? SDPA_OK : SDPA_ERR_ARCH;
+}
+
+// Tensor map over a packed bf16 [T, H, D] tensor: dims {D, H, T}, box {64, 1, rows}, 128B swizzle.
+static int make_map(CUtensorMap* map, const void* base, int T, int H, int D, int box_rows) {
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(T)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(H) * D * 2};
+    const cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = static_cast<int>(r);
+        return SDPA_ERR_CUDA;
+    }
+    return SDPA_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_common(const int32_t* cu, int B, int Hq, int Hkv, int D, float scale, int T, int max_seqlen) {
+    if (cu == nullptr) return SDPA_ERR_NULL;
+    if (B < 1 || Hq < 1 || Hkv < 1 || T < 0 || max_seqlen < 0) return SDPA_ERR_SHAPE;
+    if (D != 64 && D != 128) return SDPA_ERR_SHAPE;
+    if (Hq % Hkv != 0) return SDPA_ERR_SHAPE;
+    if (!(scale > 0.f) || !isfinite(scale)) return SDPA_ERR_SHAPE;
+    if (max_seqlen > T) return SDPA_ERR_SHAPE;
+    if (static_cast<long long>(B) * Hq > 2147483647ll) return SDPA_ERR_SHAPE;
+    return SDPA_OK;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static size_t bwd_dq_bytes(int Hq, int D, int T) { return align_up(static_cast<size_t>(T) * Hq * D * sizeof(float), 256); }
+static size_t bwd_delta_bytes(int Hq, int T) { return align_up(static_cast<size_t>(T) * Hq * sizeof(float), 256); }
+
+}  // namespace sdpa
+
+using namespace sdpa;
+
+extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, float* lse, const int32_t* cu_seqlens,
+                        int B, int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
+                        void* stream) {
+    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen);
+    if (rc != SDPA_OK) return rc;
+    if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
+    if (!q || !k || !v || !o || !lse) return SDPA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+        return SDPA_ERR_ALIGN;
+    DeviceState* st = nullptr;
+    rc = device_state(&st);
+    if (rc != SDPA_OK) return rc;
+
+    CUtensorMap mq, mk, mv;
+    if ((rc = make_map(&mq, q, total_tokens, Hq, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mk, k, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mv, v, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
+
+    FwdParams p;
+    p.cu_seqlens = cu_seqlens;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
+    p.status = st->status_ptr;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.T = total_tokens;
+    p.causal = causal ? 1 : 0;
+    p.max_seqlen = max_seqlen;
+    p.scale = scale;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    const int n_pairs = (max_seqlen + 255) / 256;
+    if (n_pairs > 65535) return SDPA_ERR_SHAPE;
+    dim3 grid(static_cast<unsigned>(B * Hq), static_cast<unsigned>(n_pairs), 1);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (D == 128)
+        sdpa_fwd_kernel<128><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, p);
+    else
+        sdpa_fwd_kernel<64><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mk, mv, p);
+    SDPA_CUDA_TRY(cudaGetLastError());
+    return SDPA_OK;
+}
+
+extern "C" size_t sdpa_bwd_workspace_bytes(int B, int Hq, int Hkv, int D, int total_tokens, int max_seqlen) {
+    if (B < 1 || Hq < 1 || Hkv < 1 || total_tokens < 0 || max_seqlen < 0 || (D != 64 && D != 128) || Hq % Hkv != 0)
+        return 0;
+    return bwd_dq_bytes(Hq, D, total_tokens) + bwd_delta_bytes(Hq, total_tokens) + 256;
+}
+
+extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
+                        void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D,
+                        int causal, float scale, int total_tokens, int max_seqlen, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen);
+    if (rc != SDPA_OK) return rc;
+    if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
+    if (!q || !k || !v || !o || !lse || !dout || !dq || !dk || !dv) return SDPA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(dout) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+        return SDPA_ERR_ALIGN;
+    const size_t need = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
+        return SDPA_ERR_WORKSPACE;
+    DeviceState* st = nullptr;
+    rc = device_state(&st);
+    if (rc != SDPA_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    float* dq_acc = static_cast<float*>(workspace);
+    float* delta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + bwd_dq_bytes(Hq, D, total_tokens));
+
+    // B0: D_i = rowsum(dO * O), and clear the fp32 dQ accumulator.
+    {
+        const long long rows = static_cast<long long>(total_tokens) * Hq;
+        const int threads = 256;
+        const int rows_per_block = threads / (D / 8);
+        const long long blocks = (rows + rows_per_block - 1) / rows_per_block;
+        if (D == 128)
+            sdpa_bwd_preprocess_kernel<128><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
+                static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
+                total_tokens, Hq);
+        else
+            sdpa_bwd_preprocess_kernel<64><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
+                static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
+                total_tokens, Hq);
+        SDPA_CUDA_TRY(cudaGetLastError());
+    }
+
+    CUtensorMap mq, mk, mv, mdo;
+    if ((rc = make_map(&mq, q, total_tokens, Hq, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mk, k, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mv, v, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mdo, dout, total_tokens, Hq, D, 128)) != SDPA_OK) return rc;
+
+    BwdParams p;
+    p.cu_seqlens = cu_seqlens;
+    p.lse = lse;
+    p.delta = delta;
+    p.dq_acc = dq_acc;
+    p.dk = static_cast<__nv_bfloat16*>(dk);
+    p.dv = static_cast<__nv_bfloat16*>(dv);
+    p.status = st->status_ptr;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.T = total_tokens;
+    p.causal = causal ? 1 : 0;
+    p.max_seqlen = max_seqlen;
+    p.scale = scale;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    const int n_kv_tiles = (max_seqlen + 127) / 128;
+    if (n_kv_tiles > 65535) return SDPA_ERR_SHAPE;
+    dim3 grid(static_cast<unsigned>(B * Hkv), static_cast<unsigned>(n_kv_tiles), 1);
+    if (D == 128)
+        sdpa_bwd_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
+    else
+        sdpa_bwd_kernel<64><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
+    SDPA_CUDA_TRY(cudaGetLastError());
+
+    // B7 (dQ part): fp32 accumulator -> bf16 with the softmax scale applied.
+    {
+        const long long n8 = static_cast<long long>(total_tokens) * Hq * D / 8;
+        const int threads = 256;
+        const long long blocks = (n8 + threads - 1) / threads;
+        sdpa_bwd_dq_convert_kernel<<<static_cast<unsigned>(blocks), threads, 0, s>>>(
+            dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale);
+        SDPA_CUDA_TRY(cudaGetLastError());
+    }
+    return SDPA_OK;
+}
+
+extern "C" int sdpa_query_status(void* stream, int* site) {
+    DeviceState* st = nullptr;
+    int rc = device_state(&st);
+    if (rc != SDPA_OK) return rc;
+    SDPA_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int word = 0;
+    SDPA_CUDA_TRY(cudaMemcpy(&word, st->status_ptr, sizeof(int), cudaMemcpyDeviceToHost));
+    if (word != 0) SDPA_CUDA_TRY(cudaMemset(st->status_ptr, 0, sizeof(int)));
+    if (site) *site = word >> 8;
+    return word & 0xff;
+}
+
+extern "C" const char* sdpa_status_string(int code) {
+    switch (code) {
+        case SDPA_OK: return "ok";
+        case SDPA_ERR_NULL: return "null pointer argument";
+        case SDPA_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case SDPA_ERR_SHAPE: return "unsupported shape or scale";
+        case SDPA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SDPA_ERR_ARCH: return "device is not compute capability 10.x";
+        case SDPA_ERR_CUDA: return "CUDA runtime or driver call failed";
+        case SDPA_STATUS_TIMEOUT: return "device-side wait timed out";
+        case SDPA_STATUS_BAD_CU_SEQLENS: return "cu_seqlens inconsistent with total_tokens/max_seqlen";
+        case SDPA_STATUS_INTERNAL: return "kernel launch precondition violated";
+        default: return "unknown code";
+    }
+}
+
+extern "C" int sdpa_last_cuda_error(void) { return tl_last_cuda_error; }
