@@ -1,0 +1,337 @@
+#!/usr/bin/env python
+"""Benchmark of the bf16 SDPA forward+backward path on B200.
+
+One "step" is one pass of the whole hot path (sdpa_fwd then sdpa_bwd) over the causal GQA
+workload c3 (B=2, Hq=32, Hkv=8, S=4096, D=128), with seeded synthetic inputs.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config c3]
+
+N > 1 (under torchrun): every rank runs the same workload on its own GPU (the path shards by
+independent (sequence, kv-head) units with no exchange step, so ranks are replicas: weak scaling);
+the timed region is bracketed by a barrier and the max over ranks is taken.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_17379_b200 import workloads as W  # noqa: E402
+
+METRIC = "SDPA fwd+bwd TFLOPS (bf16, device-timed)"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": (int(np.median(self.samples)) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_sample(w: W.Workload, inputs_bits, budget_s: float):
+    """Time the fp64 oracle (fwd+bwd) on whole (sequence, kv-head) slices of the workload until
+    about `budget_s` seconds of CPU work are done.  Returns (flops_done, seconds, n_slices, threads)."""
+    import oracle
+    qb, kb, vb, dob = inputs_bits
+    G = w.Hq // w.Hkv
+    flops = 0.0
+    secs = 0.0
+    n = 0
+    for b in range(w.B):
+        for g in range(w.Hkv):
+            r0, r1, h0, h1 = W.slice_group(w, b, g)
+            L = r1 - r0
+            if L == 0:
+                continue
+            q = W.bf16_bits_to_f64(qb[r0:r1, h0:h1])
+            k = W.bf16_bits_to_f64(kb[r0:r1, g:g + 1])
+            v = W.bf16_bits_to_f64(vb[r0:r1, g:g + 1])
+            do = W.bf16_bits_to_f64(dob[r0:r1, h0:h1])
+            t0 = time.perf_counter()
+            oracle.sdpa_bwd(q, k, v, do, np.array([0, L], np.int32), w.causal, w.scale)  # fwd is inside
+            secs += time.perf_counter() - t0
+            f = 4.0 * G * w.D * float(L) * L * (0.5 if w.causal else 1.0)
+            flops += 3.5 * f
+            n += 1
+            if secs >= budget_s:
+                return flops, secs, n, oracle.num_threads()
+    return flops, secs, n, oracle.num_threads()
+
+
+def run_reference(args, w):
+    """The fp64 CPU oracle as the reference arm: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inputs = W.make_inputs(w)
+    per_step_budget = 4.0
+    vals = []
+    for i in range(args.warmup + args.steps):
+        flops, secs, n, threads = oracle_sample(w, inputs, per_step_budget)
+        if i >= args.warmup:
+            vals.append((flops, secs, n))
+    flops = sum(v[0] for v in vals)
+    secs = sum(v[1] for v in vals)
+    value = flops / secs / 1e12
+    sample = f"{vals[0][2]} of {w.B * w.Hkv} (sequence, kv-head) slices per step, fwd+bwd, fp64"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(1, len(vals)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "fp64 CPU oracle on host cores, bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c3", choices=list(W.CONFIG_NAMES))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = W.config(args.config)
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2608_17379_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SDPA path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    binding.load()
+
+    T, Hq, Hkv, D = w.T, w.Hq, w.Hkv, w.D
+    inputs_bits = W.make_inputs(w)
+    to_t = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    host_in = [to_t(x).pin_memory() for x in inputs_bits]
+    q, k, v, do = (x.cuda() for x in host_in)
+    cu_host = torch.from_numpy(w.cu_seqlens)
+    cu = cu_host.cuda()
+    o = torch.empty_like(q)
+    lse = torch.empty((Hq, T), dtype=torch.float32, device="cuda")
+    dq = torch.empty_like(q); dk = torch.empty_like(k); dv = torch.empty_like(v)
+    ws = torch.empty(binding.sdpa_bwd_workspace_bytes(w.B, Hq, Hkv, D, T, w.max_seqlen), dtype=torch.uint8,
+                     device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def fwd():
+        binding.sdpa_fwd(q, k, v, cu, w.max_seqlen, w.causal, w.scale, o=o, lse=lse, stream=stream)
+
+    def bwd():
+        binding.sdpa_bwd(q, k, v, o, lse, do, cu, w.max_seqlen, w.causal, w.scale, dq=dq, dk=dk, dv=dv,
+                         workspace=ws, stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    ev_ms, ev_me = ev(), ev()
+    ev_ms.record(); ev_me.record()  # create the underlying CUDA events
+    for _ in range(args.warmup):
+        fwd(); bwd()
+    barrier()
+    assert binding.query_status() == (0, 0)
+
+    K = args.steps
+    e_f0 = [ev() for _ in range(K)]; e_f1 = [ev() for _ in range(K)]; e_b1 = [ev() for _ in range(K)]
+    main_ms = []
+    binding.bwd_profile_events(ev_ms, ev_me)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        t_start, t_stop = ev(), ev()
+        t_start.record()
+        for i in range(K):
+            e_f0[i].record(); fwd(); e_f1[i].record(); bwd(); e_b1[i].record()
+        t_stop.record()
+        barrier()
+    total_ms = t_start.elapsed_time(t_stop)
+    binding.bwd_profile_events(None, None)
+    # main backward kernel alone: a few extra launches with the profiling events read back each time
+    binding.bwd_profile_events(ev_ms, ev_me)
+    for _ in range(min(K, 20)):
+        bwd(); torch.cuda.synchronize(); main_ms.append(ev_ms.elapsed_time(ev_me))
+    binding.bwd_profile_events(None, None)
+    status = binding.query_status()
+    assert status == (0, 0), status
+
+    fwd_ms = float(np.median([e_f0[i].elapsed_time(e_f1[i]) for i in range(K)]))
+    bwd_ms = float(np.median([e_f1[i].elapsed_time(e_b1[i]) for i in range(K)]))
+    step_ms = total_ms / K
+    if dist is not None:
+        t = torch.tensor([step_ms, fwd_ms, bwd_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms, fwd_ms, bwd_ms = (float(x) for x in t.tolist())
+
+    # ---- end to end through the C ABI with HOST buffers (copies inside the timed region)
+    o_h = torch.empty((T, Hq, D), dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty((Hq, T), dtype=torch.float32).pin_memory()
+    dq_h = torch.empty_like(o_h).pin_memory()
+    dk_h = torch.empty((T, Hkv, D), dtype=torch.bfloat16).pin_memory(); dv_h = torch.empty_like(dk_h).pin_memory()
+    staging = torch.empty(binding.sdpa_host_staging_bytes(w.B, Hq, Hkv, D, T, w.max_seqlen), dtype=torch.uint8,
+                          device="cuda")
+
+    def e2e_step():
+        binding.sdpa_fwd_bwd_host(host_in[0], host_in[1], host_in[2], host_in[3], o_h, lse_h, dq_h, dk_h, dv_h,
+                                  cu_host, w.max_seqlen, w.causal, w.scale, staging, stream=stream)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    Ke = max(3, min(K, 10))
+    s0, s1 = ev(), ev()
+    s0.record()
+    for _ in range(Ke):
+        e2e_step()
+    s1.record()
+    barrier()
+    e2e_ms = s0.elapsed_time(s1) / Ke
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    assert binding.query_status() == (0, 0)
+    h2d = 2 * (T * Hq * D * 2) + 2 * (T * Hkv * D * 2) + (w.B + 1) * 4
+    d2h = 2 * (T * Hq * D * 2) + 2 * (T * Hkv * D * 2) + T * Hq * 4
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    step_flops = w.fwd_flops() + w.bwd_flops()
+    value = world * step_flops / (step_ms * 1e-3) / 1e12
+    fwd_tf = w.fwd_flops() / (fwd_ms * 1e-3) / 1e12
+    bwd_tf = w.bwd_flops() / (bwd_ms * 1e-3) / 1e12
+    main_med = float(np.median(main_ms))
+    main_tf = w.bwd_flops() / (main_med * 1e-3) / 1e12
+    peak = float(peaks["bf16_tflops"])
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{w.name}: causal={w.causal} B={w.B} Hq={Hq} Hkv={Hkv} S={w.max_seqlen} D={D}",
+                   "seed": w.seed, "total_tokens": T,
+                   "l2": "inputs+outputs+workspace of a step (>500 MB) exceed the 126 MB L2; no flush",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "fwd": {"ms": fwd_ms, "tflops": fwd_tf, "frac_of_measured_burst": fwd_tf / peak,
+                "frac_of_measured_sustained": fwd_tf / float(peaks["bf16_tflops_sustained"]),
+                "frac_of_nominal_2250": fwd_tf / NOMINAL_BF16_TFLOPS},
+        "bwd": {"ms": bwd_ms, "tflops": bwd_tf, "frac_of_measured_burst": bwd_tf / peak,
+                "frac_of_measured_sustained": bwd_tf / float(peaks["bf16_tflops_sustained"]),
+                "frac_of_nominal_2250": bwd_tf / NOMINAL_BF16_TFLOPS, "kernels": 3},
+        "roofline": {"bound": "tensor", "kernel": "sdpa_bwd_kernel<128>", "achieved": main_tf, "peak": peak,
+                     "unit": "TFLOP/s", "frac": main_tf / peak, "peak_source": f"{peaks['_source']} bf16 burst",
+                     "ms_per_launch": main_med, "flops_per_launch": w.bwd_flops(), "traffic": None,
+                     "fwd_kernel": {"kernel": "sdpa_fwd_kernel<128>", "achieved": fwd_tf, "frac": fwd_tf / peak,
+                                    "ms_per_launch": fwd_ms, "flops_per_launch": w.fwd_flops()},
+                     "hbm_min_bytes_per_step": w.min_bytes_fwd() + w.min_bytes_bwd(),
+                     "hbm_gbs_at_min_bytes": (w.min_bytes_fwd() + w.min_bytes_bwd()) / (step_ms * 1e-3) / 1e9,
+                     "hbm_peak_gbs": float(peaks["hbm_gbs"])},
+        "e2e": {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "sdpa_fwd_bwd_host (pinned host buffers)"},
+        "gpu_launches": 4 * K,
+        "clocks": clocks.summary(),
+    }
+    if not args.no_cpu_baseline:
+        flops, secs, n, threads = oracle_sample(w, inputs_bits, 12.0)
+        line["cpu_baseline"] = {"value": flops / secs / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+                                "sample": f"{n} of {w.B * w.Hkv} (sequence, kv-head) slices of {w.name}, fwd+bwd fp64, "
+                                          f"{secs:.1f} s"}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -94,6 +94,30 @@ int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Whole step with HOST buffers (no counterpart in the paper's operator list beyond composing the
+ * forward and backward workloads of its appendix "Workloads"): copies q, k, v, dout and cu_seqlens
+ * from host memory to the device, runs sdpa_fwd then sdpa_bwd, and copies o, lse, dq, dk, dv back,
+ * all asynchronously on `stream`.  Host pointers should be page-locked for the copies to overlap;
+ * layouts are those of sdpa_fwd / sdpa_bwd.  `staging` is caller-owned, 256-byte aligned DEVICE
+ * scratch of at least sdpa_host_staging_bytes(...) bytes that holds the device copies and the
+ * backward workspace; the library allocates nothing.  The host outputs are valid once the stream
+ * has been synchronised.
+ */
+size_t sdpa_host_staging_bytes(int B, int Hq, int Hkv, int D, int total_tokens, int max_seqlen);
+int sdpa_fwd_bwd_host(const void* q, const void* k, const void* v, const void* dout, void* o,
+                      float* lse, void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B,
+                      int Hq, int Hkv, int D, int causal, float scale, int total_tokens,
+                      int max_seqlen, void* staging, size_t staging_bytes, void* stream);
+
+/*
+ * Profiling hook (measurement protocol of the paper's section "Multi-turn Evaluation Protocol":
+ * per-kernel device timing): registers, for the calling thread, two caller-owned cudaEvent_t that
+ * every later sdpa_bwd records on its stream immediately before and after its main kernel (between
+ * the D_i preprocess and the dQ conversion).  Pass null pointers to switch it off.  Returns SDPA_OK.
+ */
+int sdpa_bwd_profile_events(void* ev_main_start, void* ev_main_stop);
+
+/*
  * Waits for `stream`, then returns the current device's status word (0 = no device-side problem
  * since the last query; otherwise an SDPA_STATUS_* code) and clears it.  *site (may be null)
  * receives an internal identifier of the wait that gave up.  Returns SDPA_ERR_CUDA if the

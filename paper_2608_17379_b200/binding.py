@@ -17,7 +17,8 @@ _LIB = None
 
 SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
-           "sdpa_status_string", "sdpa_last_cuda_error")
+           "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
+           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events")
 
 
 class SdpaError(RuntimeError):
@@ -40,6 +41,12 @@ def load():
     lib.sdpa_bwd_workspace_bytes.argtypes = [ci] * 6
     lib.sdpa_bwd.restype = ci
     lib.sdpa_bwd.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp, ctypes.c_size_t, vp]
+    lib.sdpa_host_staging_bytes.restype = ctypes.c_size_t
+    lib.sdpa_host_staging_bytes.argtypes = [ci] * 6
+    lib.sdpa_fwd_bwd_host.restype = ci
+    lib.sdpa_fwd_bwd_host.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp, ctypes.c_size_t, vp]
+    lib.sdpa_bwd_profile_events.restype = ci
+    lib.sdpa_bwd_profile_events.argtypes = [vp, vp]
     lib.sdpa_query_status.restype = ci
     lib.sdpa_query_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.sdpa_status_string.restype = ctypes.c_char_p
@@ -119,6 +126,34 @@ def sdpa_bwd(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, s
                       _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
     _check(rc, "sdpa_bwd")
     return dq, dk, dv
+
+
+def sdpa_host_staging_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen) -> int:
+    return int(load().sdpa_host_staging_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen))
+
+
+def sdpa_fwd_bwd_host(q, k, v, dout, o, lse, dq, dk, dv, cu_seqlens, max_seqlen: int, causal: bool, scale: float,
+                      staging, stream=None):
+    """Whole step on HOST tensors (pinned CPU torch tensors in, pinned CPU tensors out); ``staging``
+    is a CUDA uint8 tensor of at least sdpa_host_staging_bytes(...) bytes.  Asynchronous."""
+    lib = load()
+    for t in (q, k, v, dout, o, lse, dq, dk, dv, cu_seqlens):
+        assert not t.is_cuda and t.is_contiguous()
+    assert staging.is_cuda
+    T, Hq, Hkv, D = _dims(q, k)
+    B = cu_seqlens.numel() - 1
+    rc = lib.sdpa_fwd_bwd_host(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(o), _ptr(lse), _ptr(dq), _ptr(dk),
+                               _ptr(dv), _ptr(cu_seqlens), B, Hq, Hkv, D, int(bool(causal)), float(scale), T,
+                               int(max_seqlen), _ptr(staging), int(staging.numel()), _stream_ptr(stream))
+    _check(rc, "sdpa_fwd_bwd_host")
+
+
+def bwd_profile_events(start=None, stop=None):
+    """Register two recorded-at-least-once torch.cuda.Event objects to be recorded around the main
+    backward kernel by later sdpa_bwd calls of this thread (None, None switches it off)."""
+    s = 0 if start is None else int(start.cuda_event)
+    e = 0 if stop is None else int(stop.cuda_event)
+    _check(load().sdpa_bwd_profile_events(s, e), "sdpa_bwd_profile_events")
 
 
 def query_status(stream=None):

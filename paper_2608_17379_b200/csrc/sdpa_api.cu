@@ -18,6 +18,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static thread_local int tl_last_cuda_error = 0;
+// Optional caller-owned events recorded around the main backward kernel (profiling hook).
+static thread_local cudaEvent_t tl_ev_main_start = nullptr;
+static thread_local cudaEvent_t tl_ev_main_stop = nullptr;
 
 #define SDPA_CUDA_TRY(expr)                          \
     do {                                             \
@@ -226,11 +229,13 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
     const int n_kv_tiles = (max_seqlen + 127) / 128;
     if (n_kv_tiles > 65535) return SDPA_ERR_SHAPE;
     dim3 grid(static_cast<unsigned>(B * Hkv), static_cast<unsigned>(n_kv_tiles), 1);
+    if (tl_ev_main_start) SDPA_CUDA_TRY(cudaEventRecord(tl_ev_main_start, s));
     if (D == 128)
         sdpa_bwd_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
     else
         sdpa_bwd_kernel<64><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
     SDPA_CUDA_TRY(cudaGetLastError());
+    if (tl_ev_main_stop) SDPA_CUDA_TRY(cudaEventRecord(tl_ev_main_stop, s));
 
     // B7 (dQ part): fp32 accumulator -> bf16 with the softmax scale applied.
     {
@@ -241,6 +246,63 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
             dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale);
         SDPA_CUDA_TRY(cudaGetLastError());
     }
+    return SDPA_OK;
+}
+
+extern "C" int sdpa_bwd_profile_events(void* ev_main_start, void* ev_main_stop) {
+    tl_ev_main_start = static_cast<cudaEvent_t>(ev_main_start);
+    tl_ev_main_stop = static_cast<cudaEvent_t>(ev_main_stop);
+    return SDPA_OK;
+}
+
+extern "C" size_t sdpa_host_staging_bytes(int B, int Hq, int Hkv, int D, int total_tokens, int max_seqlen) {
+    const size_t ws = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
+    if (ws == 0) return 0;
+    const size_t T = static_cast<size_t>(total_tokens);
+    const size_t qb = align_up(T * Hq * D * 2, 256), kb = align_up(T * Hkv * D * 2, 256);
+    const size_t lb = align_up(T * Hq * 4, 256), cb = align_up(static_cast<size_t>(B + 1) * 4, 256);
+    return 4 * qb /* q, o, dout, dq */ + 4 * kb /* k, v, dk, dv */ + lb + cb + ws;
+}
+
+extern "C" int sdpa_fwd_bwd_host(const void* q, const void* k, const void* v, const void* dout, void* o, float* lse,
+                                 void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv,
+                                 int D, int causal, float scale, int total_tokens, int max_seqlen, void* staging,
+                                 size_t staging_bytes, void* stream) {
+    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen);
+    if (rc != SDPA_OK) return rc;
+    if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
+    if (!q || !k || !v || !dout || !o || !lse || !dq || !dk || !dv) return SDPA_ERR_NULL;
+    const size_t need = sdpa_host_staging_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
+    if (staging == nullptr || (reinterpret_cast<uintptr_t>(staging) & 255u) || staging_bytes < need)
+        return SDPA_ERR_WORKSPACE;
+    const size_t T = static_cast<size_t>(total_tokens);
+    const size_t q_bytes = T * Hq * D * 2, k_bytes = T * Hkv * D * 2, l_bytes = T * Hq * 4;
+    const size_t c_bytes = static_cast<size_t>(B + 1) * 4;
+    const size_t qb = align_up(q_bytes, 256), kb = align_up(k_bytes, 256);
+    const size_t lb = align_up(l_bytes, 256), cb = align_up(c_bytes, 256);
+    uint8_t* base = static_cast<uint8_t*>(staging);
+    uint8_t* d_q = base;            uint8_t* d_o = d_q + qb;   uint8_t* d_do = d_o + qb;  uint8_t* d_dq = d_do + qb;
+    uint8_t* d_k = d_dq + qb;       uint8_t* d_v = d_k + kb;   uint8_t* d_dk = d_v + kb;  uint8_t* d_dv = d_dk + kb;
+    uint8_t* d_lse = d_dv + kb;     uint8_t* d_cu = d_lse + lb; uint8_t* d_ws = d_cu + cb;
+    const size_t ws_bytes = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    SDPA_CUDA_TRY(cudaMemcpyAsync(d_cu, cu_seqlens, c_bytes, cudaMemcpyHostToDevice, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(d_q, q, q_bytes, cudaMemcpyHostToDevice, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(d_k, k, k_bytes, cudaMemcpyHostToDevice, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(d_v, v, k_bytes, cudaMemcpyHostToDevice, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(d_do, dout, q_bytes, cudaMemcpyHostToDevice, s));
+    rc = sdpa_fwd(d_q, d_k, d_v, d_o, reinterpret_cast<float*>(d_lse), reinterpret_cast<const int32_t*>(d_cu), B, Hq,
+                  Hkv, D, causal, scale, total_tokens, max_seqlen, stream);
+    if (rc != SDPA_OK) return rc;
+    rc = sdpa_bwd(d_q, d_k, d_v, d_o, reinterpret_cast<const float*>(d_lse), d_do, d_dq, d_dk, d_dv,
+                  reinterpret_cast<const int32_t*>(d_cu), B, Hq, Hkv, D, causal, scale, total_tokens, max_seqlen, d_ws,
+                  ws_bytes, stream);
+    if (rc != SDPA_OK) return rc;
+    SDPA_CUDA_TRY(cudaMemcpyAsync(o, d_o, q_bytes, cudaMemcpyDeviceToHost, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(lse, d_lse, l_bytes, cudaMemcpyDeviceToHost, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(dq, d_dq, q_bytes, cudaMemcpyDeviceToHost, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(dk, d_dk, k_bytes, cudaMemcpyDeviceToHost, s));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(dv, d_dv, k_bytes, cudaMemcpyDeviceToHost, s));
     return SDPA_OK;
 }
 

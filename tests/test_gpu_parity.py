@@ -1,0 +1,247 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle.
+
+Tolerances are those of the benchmark definition: max|O-O*| <= 2e-2, max|LSE-LSE*| <= 1e-3,
+max|dX-dX*|/max|dX*| <= 5e-2 for dQ, dK, dV (bf16 path against the unrounded oracle).
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import sdpa_testlib as TL
+from paper_2608_17379_b200 import binding
+from paper_2608_17379_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_compare(w, slices=None, bwd=True):
+    inputs = W.make_inputs(w)
+    out = TL.run_gpu(*inputs, w.cu_seqlens, w.max_seqlen, w.causal, w.scale, bwd=bwd)
+    worst = TL.compare_slices(w, inputs, out, slices if slices is not None else TL.all_slices(w))
+    TL.assert_within(worst, bwd=bwd)
+    return worst, out
+
+
+# ------------------------------------------------------------------ small shapes, element by element
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("lengths,Hq,Hkv,D", [
+    ((128,), 2, 2, 64),            # c1 shape
+    ((1,), 1, 1, 128),             # single token
+    ((127,), 2, 1, 128),           # one short tile
+    ((129,), 2, 2, 128),           # one row into the second tile
+    ((256,), 1, 1, 128),           # exactly one tile pair
+    ((257,), 2, 1, 64),
+    ((640,), 4, 2, 128),           # several tiles, odd tile count
+    ((300, 77, 513), 4, 2, 128),   # packed, ragged, GQA
+    ((0, 5, 0, 260, 0), 2, 1, 64),  # empty sequences in the batch
+    ((1000,), 8, 1, 128),          # G = 8
+])
+def test_small_shapes(lengths, Hq, Hkv, D, causal):
+    w = TL.random_workload(lengths, Hq, Hkv, D, causal, seed=100 + len(lengths) + Hq)
+    run_and_compare(w)
+
+
+def test_config_c1_full():
+    run_and_compare(W.config("c1"))
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_every_length_up_to_260(causal):
+    """One head, D=64: every sequence length 1..260 (tile boundaries at 128 and 256)."""
+    worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dk": 0.0, "dv": 0.0}
+    for L in range(1, 261):
+        w = TL.random_workload((L,), 1, 1, 64, causal, seed=1000 + L)
+        inputs = W.make_inputs(w)
+        out = TL.run_gpu(*inputs, w.cu_seqlens, w.max_seqlen, w.causal, w.scale)
+        e = TL.compare_slices(w, inputs, out, [(0, 0)])
+        for k in worst:
+            worst[k] = max(worst[k], e[k])
+    TL.assert_within(worst)
+
+
+def test_paper_ragged_shape():
+    """The paper's ragged GQA prefill shape: 33 sequences, 16,294 tokens, 32 query / 4 kv heads,
+    D=128, causal (lengths are synthetic; the original records are not available)."""
+    rng = np.random.default_rng(33)
+    cuts = np.sort(rng.choice(np.arange(1, 16294), 32, replace=False))
+    lengths = np.diff(np.concatenate([[0], cuts, [16294]]))
+    assert lengths.sum() == 16294 and len(lengths) == 33
+    w = TL.random_workload([int(x) for x in lengths], 32, 4, 128, True, seed=33)
+    order = np.argsort(lengths)
+    slices = [(int(order[-1]), 0), (int(order[0]), 3), (int(order[16]), 1)]
+    run_and_compare(w, slices)
+
+
+# ------------------------------------------------------------------ full-size configurations, sampled slices
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c4c", "c5"])
+def test_full_configs_on_sampled_slices(name):
+    """The five benchmark configurations in the launch configuration the bench times; the oracle
+    checks complete O/LSE/dQ/dK/dV of independent (sequence, kv-head) slices."""
+    w = W.config(name)
+    if name == "c5":
+        lens = np.array(w.lengths)
+        slices = [(int(np.argmin(lens)), 0), (int(np.argsort(lens)[len(lens) // 2]), w.Hkv - 1)]
+    elif name in ("c4", "c4c"):
+        slices = [(0, 5)]
+    else:
+        slices = [(0, 0), (w.B - 1, w.Hkv - 1)]
+    run_and_compare(w, slices)
+
+
+# ------------------------------------------------------------------ numerically hard inputs
+def _custom(q, k, v, do, lengths, causal, scale):
+    """float64 arrays -> bf16 bits -> GPU and oracle; returns worst errors."""
+    bits = [W.f32_to_bf16_bits(x.astype(np.float32)) for x in (q, k, v, do)]
+    T, Hq, D = q.shape
+    w = W.Workload("custom", 0, tuple(lengths), Hq, k.shape[1], D, causal)
+    out = TL.run_gpu(*bits, w.cu_seqlens, w.max_seqlen, causal, scale)
+    return TL.compare_slices(w, bits, out, TL.all_slices(w)), w
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_row_max_grows_with_key_index(causal):
+    """Scores increase along the key axis, so every key tile raises the running max and forces a
+    rescale of the accumulated output (a kernel that treats tiles independently fails here)."""
+    L, D = 1024, 128
+    rng = np.random.default_rng(5)
+    u = rng.standard_normal(D); u /= np.linalg.norm(u)
+    q = rng.standard_normal((L, 2, D)) * 0.3 + 4.0 * u
+    k = rng.standard_normal((L, 2, D)) * 0.3 + (np.arange(L)[:, None, None] / L * 60.0) * u
+    v = rng.standard_normal((L, 2, D)); do = rng.standard_normal((L, 2, D))
+    worst, _ = _custom(q, k, v, do, [L], causal, 1.0 / np.sqrt(D))
+    TL.assert_within(worst)
+
+
+def test_large_score_magnitudes_do_not_overflow():
+    """Scaled scores around +-60..100: a missing max subtraction would overflow exp."""
+    L, D = 384, 64
+    rng = np.random.default_rng(6)
+    q = rng.standard_normal((L, 1, D)) * 6.0
+    k = rng.standard_normal((L, 1, D)) * 6.0
+    v = rng.standard_normal((L, 1, D)); do = rng.standard_normal((L, 1, D))
+    s = (q[:, 0] @ k[:, 0].T) / np.sqrt(D)
+    assert np.abs(s).max() > 60
+    worst, _ = _custom(q, k, v, do, [L], False, 1.0 / np.sqrt(D))
+    TL.assert_within(worst)
+
+
+def test_constant_v_and_causal_row0_on_gpu():
+    w = TL.random_workload((300, 140), 4, 2, 128, True, seed=77)
+    qb, kb, vb, dob = W.make_inputs(w)
+    c = W.gen_tensor_bits(78, W.TENSOR_V, (1, w.Hkv, w.D))
+    vb = np.broadcast_to(c, vb.shape).copy()
+    out = TL.run_gpu(qb, kb, vb, dob, w.cu_seqlens, w.max_seqlen, True, w.scale, bwd=False)
+    o = TL.to_f64(out["o"])
+    cf = W.bf16_bits_to_f64(c)
+    G = w.Hq // w.Hkv
+    for h in range(w.Hq):
+        assert np.max(np.abs(o[:, h] - cf[0, h // G])) <= 2e-2
+    # causal row 0 of each sequence: O = V row 0 exactly (P = 1), LSE = s_00
+    q = W.bf16_bits_to_f64(qb); k = W.bf16_bits_to_f64(kb)
+    lse = TL.to_f64(out["lse"])
+    for b in range(w.B):
+        r = int(w.cu_seqlens[b])
+        for h in range(w.Hq):
+            assert abs(lse[h, r] - w.scale * q[r, h] @ k[r, h // G]) <= 1e-3
+
+
+# ------------------------------------------------------------------ determinism, isolation of the backward
+def test_forward_is_bit_reproducible():
+    w = TL.random_workload((700, 300), 4, 2, 128, True, seed=55)
+    inputs = W.make_inputs(w)
+    a = TL.run_gpu(*inputs, w.cu_seqlens, w.max_seqlen, True, w.scale, bwd=False)
+    b = TL.run_gpu(*inputs, w.cu_seqlens, w.max_seqlen, True, w.scale, bwd=False)
+    assert torch.equal(a["o"].view(torch.int16), b["o"].view(torch.int16))
+    assert torch.equal(a["lse"].view(torch.int32), b["lse"].view(torch.int32))
+
+
+def test_dk_dv_are_bit_reproducible_and_dq_is_close():
+    w = TL.random_workload((700, 300), 4, 2, 128, True, seed=56)
+    inputs = W.make_inputs(w)
+    a = TL.run_gpu(*inputs, w.cu_seqlens, w.max_seqlen, True, w.scale)
+    b = TL.run_gpu(*inputs, w.cu_seqlens, w.max_seqlen, True, w.scale)
+    assert torch.equal(a["dk"].view(torch.int16), b["dk"].view(torch.int16))
+    assert torch.equal(a["dv"].view(torch.int16), b["dv"].view(torch.int16))
+    d = (a["dq"].float() - b["dq"].float()).abs().max().item()
+    assert d <= 2e-2 * a["dq"].float().abs().max().item()  # atomics: order of fp32 additions may differ
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_fed_with_oracle_forward(causal):
+    """Backward alone: O (rounded to bf16) and LSE (rounded to fp32) come from the oracle."""
+    w = TL.random_workload((500,), 4, 2, 128, causal, seed=57)
+    qb, kb, vb, dob = W.make_inputs(w)
+    q, k, v, do = (W.bf16_bits_to_f64(x) for x in (qb, kb, vb, dob))
+    dq, dk, dv, o, lse = oracle.sdpa_bwd(q, k, v, do, w.cu_seqlens, causal, w.scale)
+    dev = [TL.to_dev(x) for x in (qb, kb, vb, dob)]
+    o_d = TL.to_dev(W.f32_to_bf16_bits(o.astype(np.float32)))
+    lse_d = torch.from_numpy(lse.astype(np.float32)).cuda()
+    cu_d = torch.from_numpy(w.cu_seqlens).cuda()
+    gdq, gdk, gdv = binding.sdpa_bwd(dev[0], dev[1], dev[2], o_d, lse_d, dev[3], cu_d, w.max_seqlen, causal, w.scale)
+    assert binding.query_status() == (0, 0)
+    for got, ref in ((gdq, dq), (gdk, dk), (gdv, dv)):
+        assert np.max(np.abs(TL.to_f64(got) - ref)) / np.max(np.abs(ref)) <= TL.TOL_GRAD
+
+
+def test_outputs_outside_the_batch_are_untouched():
+    """Canaries around the outputs and the workspace: nothing outside the tensors is written."""
+    w = TL.random_workload((130, 61), 2, 1, 128, True, seed=58)
+    qb, kb, vb, dob = W.make_inputs(w)
+    q, k, v, do = (TL.to_dev(x) for x in (qb, kb, vb, dob))
+    cu = torch.from_numpy(w.cu_seqlens).cuda()
+    T, Hq, Hkv, D = w.T, w.Hq, w.Hkv, w.D
+    pad = 4096
+
+    def guarded(nbytes):
+        buf = torch.full((nbytes + 2 * pad,), 0x5A, dtype=torch.uint8, device="cuda")
+        return buf, buf[pad:pad + nbytes]
+
+    bo, o = guarded(T * Hq * D * 2); bl, lse = guarded(Hq * T * 4)
+    bq, dq = guarded(T * Hq * D * 2); bk, dk = guarded(T * Hkv * D * 2); bv, dv = guarded(T * Hkv * D * 2)
+    need = binding.sdpa_bwd_workspace_bytes(w.B, Hq, Hkv, D, T, w.max_seqlen)
+    bw, ws = guarded(need)
+    o_t = o.view(torch.bfloat16).view(T, Hq, D); lse_t = lse.view(torch.float32).view(Hq, T)
+    binding.sdpa_fwd(q, k, v, cu, w.max_seqlen, True, w.scale, o=o_t, lse=lse_t)
+    binding.sdpa_bwd(q, k, v, o_t, lse_t, do, cu, w.max_seqlen, True, w.scale,
+                     dq=dq.view(torch.bfloat16).view(T, Hq, D), dk=dk.view(torch.bfloat16).view(T, Hkv, D),
+                     dv=dv.view(torch.bfloat16).view(T, Hkv, D), workspace=ws)
+    assert binding.query_status() == (0, 0)
+    for buf in (bo, bl, bq, bk, bv, bw):
+        assert bool((buf[:pad] == 0x5A).all()) and bool((buf[-pad:] == 0x5A).all())
+
+
+# ------------------------------------------------------------------ boundary behaviour on the device
+def test_bad_cu_seqlens_is_reported_not_faulted():
+    w = TL.random_workload((200,), 2, 2, 64, False, seed=59)
+    qb, kb, vb, dob = W.make_inputs(w)
+    q, k, v = (TL.to_dev(x) for x in (qb, kb, vb))
+    cu = torch.tensor([0, 100000], dtype=torch.int32, device="cuda")  # contradicts total_tokens = 200
+    binding.sdpa_fwd(q, k, v, cu, w.max_seqlen, False, w.scale)
+    st, _ = binding.query_status()
+    assert st == 2
+    assert binding.query_status() == (0, 0)  # cleared by the query
+
+
+def test_host_buffer_entry_point_matches_device_entry_points():
+    w = TL.random_workload((333, 200), 4, 2, 128, True, seed=60)
+    qb, kb, vb, dob = W.make_inputs(w)
+    ref = TL.run_gpu(qb, kb, vb, dob, w.cu_seqlens, w.max_seqlen, True, w.scale)
+    host = [torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in (qb, kb, vb, dob)]
+    T, Hq, Hkv, D = w.T, w.Hq, w.Hkv, w.D
+    o = torch.empty((T, Hq, D), dtype=torch.bfloat16).pin_memory()
+    lse = torch.empty((Hq, T), dtype=torch.float32).pin_memory()
+    dq = torch.empty_like(o).pin_memory()
+    dk = torch.empty((T, Hkv, D), dtype=torch.bfloat16).pin_memory(); dv = torch.empty_like(dk).pin_memory()
+    staging = torch.empty(binding.sdpa_host_staging_bytes(w.B, Hq, Hkv, D, T, w.max_seqlen), dtype=torch.uint8,
+                          device="cuda")
+    binding.sdpa_fwd_bwd_host(host[0], host[1], host[2], host[3], o, lse, dq, dk, dv, torch.from_numpy(w.cu_seqlens),
+                              w.max_seqlen, True, w.scale, staging)
+    assert binding.query_status() == (0, 0)
+    assert torch.equal(o.view(torch.int16), ref["o"].cpu().view(torch.int16))
+    assert torch.equal(lse, ref["lse"].cpu())
+    assert torch.equal(dk.view(torch.int16), ref["dk"].cpu().view(torch.int16))
+    assert torch.equal(dv.view(torch.int16), ref["dv"].cpu().view(torch.int16))
+    assert (dq.float() - ref["dq"].cpu().float()).abs().max() <= 2e-2 * ref["dq"].float().abs().max().item()
