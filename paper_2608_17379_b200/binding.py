@@ -12,7 +12,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsdpa_b200.so")
+LIB_PATH = os.environ.get("SDPA_B200_LIB", os.path.join(_HERE, "libsdpa_b200.so"))
 _LIB = None
 
 SDPA_OK = 0

@@ -230,7 +230,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (valid) p.lse[static_cast<size_t>(h) * p.T + r0 + row] = m * p.scale + logf(l);
         }
     } else {
-        setmaxnreg_dec<40>();
+        setmaxnreg_dec<80>();
         if (warp == 9) {
             // -------------------------------------------------------- TMA producer
             if (elect_one()) {
@@ -266,26 +266,31 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (elect_one()) {
                 constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
                 constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, false, true);
-                const uint32_t q_addr = smem_u32(sQ);
-                const uint32_t ring_addr = smem_u32(sRing);
+                // The issuing thread's own instruction stream bounds the MMA rate (every extra ALU
+                // instruction between two tcgen05.mma costs several cycles), so descriptors are built
+                // once and only advanced by constants inside the loops.
+                const uint64_t q_desc0 = smem_desc_sw128(smem_u32(sQ), 0, 1024);
+                const uint64_t q_desc1 = smem_desc_sw128(smem_u32(sQ) + Cfg::kTileBytes, 0, 1024);
+                const uint64_t k_desc = smem_desc_sw128(smem_u32(sRing), 0, 1024);                 // K-major
+                const uint64_t v_desc = smem_desc_sw128(smem_u32(sRing), Cfg::kAtomBytes, 1024);  // MN-major
                 auto issue_qk = [&](int t, int st) {
-                    const uint32_t a0 = q_addr + t * Cfg::kTileBytes;
-                    const uint32_t b0 = ring_addr + st * Cfg::kTileBytes;
+                    const uint64_t a0 = t == 0 ? q_desc0 : q_desc1;
+                    const uint64_t b0 = k_desc + static_cast<uint64_t>(st * (Cfg::kTileBytes >> 4));
+                    const uint32_t d = tmem + t * 128;
 #pragma unroll
                     for (int kk = 0; kk < Cfg::kKSteps; ++kk) {
-                        const uint32_t off = (kk >> 2) * Cfg::kAtomBytes + (kk & 3) * 32;
-                        umma_ss(tmem + t * 128, smem_desc_sw128(a0 + off, 0, 1024), smem_desc_sw128(b0 + off, 0, 1024),
-                                idesc_qk, kk > 0);
+                        const uint64_t off = static_cast<uint64_t>(((kk >> 2) * Cfg::kAtomBytes + (kk & 3) * 32) >> 4);
+                        umma_ss(d, a0 + off, b0 + off, idesc_qk, kk > 0);
                     }
                 };
                 auto issue_pv = [&](int t, int st, bool accumulate) {
-                    const uint32_t b0 = ring_addr + st * Cfg::kTileBytes;
+                    const uint64_t b0 = v_desc + static_cast<uint64_t>(st * (Cfg::kTileBytes >> 4));
+                    const uint32_t d = tmem + 256 + t * 128;
+                    const uint32_t a = tmem + t * 128;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        umma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
-                                smem_desc_sw128(b0 + kk * 2048, Cfg::kAtomBytes, 1024), idesc_pv,
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(d, a + kk * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_pv,
                                 (accumulate || kk > 0) ? 1u : 0u);
-                    }
                 };
                 bool ok = true;
                 int it = 0;  // ring consumer counter: K_j is item 2j, V_j is item 2j+1

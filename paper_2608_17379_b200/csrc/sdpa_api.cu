@@ -208,10 +208,10 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
     }
 
     CUtensorMap mq, mk, mv, mdo;
-    if ((rc = make_map(&mq, q, total_tokens, Hq, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mq, q, total_tokens, Hq, D, 64)) != SDPA_OK) return rc;
     if ((rc = make_map(&mk, k, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
     if ((rc = make_map(&mv, v, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mdo, dout, total_tokens, Hq, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mdo, dout, total_tokens, Hq, D, 64)) != SDPA_OK) return rc;
 
     BwdParams p;
     p.cu_seqlens = cu_seqlens;
@@ -243,7 +243,7 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
         const int threads = 256;
         const long long blocks = (n8 + threads - 1) / threads;
         sdpa_bwd_dq_convert_kernel<<<static_cast<unsigned>(blocks), threads, 0, s>>>(
-            dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale);
+            dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale, total_tokens, Hq, D);
         SDPA_CUDA_TRY(cudaGetLastError());
     }
     return SDPA_OK;
