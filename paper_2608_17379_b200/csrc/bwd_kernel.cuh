@@ -26,6 +26,17 @@
 
 namespace sdpa {
 
+#ifdef SDPA_TRACE
+__device__ long long g_trace[5 * 32 * 8];
+#define SDPA_TR(role, it, k)                                                                   \
+    do {                                                                                       \
+        if (blockIdx.x == 0 && blockIdx.y == 4 && (it) >= 8 && (it) < 40)                       \
+            g_trace[((role) * 32 + ((it) - 8)) * 8 + (k)] = clock64();                         \
+    } while (0)
+#else
+#define SDPA_TR(role, it, k) do { } while (0)
+#endif
+
 struct BwdParams {
     const int32_t* cu_seqlens;
     const float* lse;    // [Hq, T]
@@ -241,7 +252,9 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = true;
         // A(s): P^T = exp2(S^T * scale_log2 - lse2) with masks; bf16 P^T overwrites the S^T columns
         auto stage_a = [&](int s) -> bool {
+            if (tid == 0) SDPA_TR(0, s - 1, 4);
             if (!mbar_wait_warp(&s_full[s & 1], (s >> 1) & 1, ctl, kBSiteSFull)) return false;
+            if (tid == 0) SDPA_TR(0, s - 1, 5);
             tc_fence_after();
             const int q0 = (i_start + s % per_head) * 64;
             const uint32_t tS = tmem + lane_base + kColS + (s & 1) * 64 + wg * 32;
@@ -276,11 +289,14 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&p_ready[s & 1]);
+            if (tid == 0) SDPA_TR(0, s - 1, 6);
             return true;
         };
         // B(s): dS^T = P^T * (dP^T - D_i) -> bf16 -> swizzled shared memory
         auto stage_b = [&](int s) -> bool {
+            if (tid == 0) SDPA_TR(0, s, 0);
             if (!mbar_wait_warp(&dp_full[s & 1], (s >> 1) & 1, ctl, kBSiteDpFull)) return false;
+            if (tid == 0) SDPA_TR(0, s, 1);
             tc_fence_after();
             const uint32_t tDP = tmem + lane_base + kColDP + (s & 1) * 64 + wg * 32;
             const float4* dl4 = reinterpret_cast<const float4*>(sRows + (s & 1) * 128 + 64 + wg * 32);
@@ -298,6 +314,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (s >= 2) {
                 if (!mbar_wait_warp(&ds_free[s & 1], ((s >> 1) - 1) & 1, ctl, kBSiteDsFree)) return false;
             }
+            if (tid == 0) SDPA_TR(0, s, 2);
             uint8_t* ds_buf = sDS + (s & 1) * 16384;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
@@ -311,6 +328,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(&ds_ready[s & 1]);
+            if (tid == 0) SDPA_TR(0, s, 3);
             return true;
         };
 
@@ -365,8 +383,10 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int it = 0; it < n_it && ok; ++it) {
             const int h = g * G + it / per_head;
             const int q0 = (i_start + it % per_head) * 64;
+            if (x == 0) SDPA_TR(4, it, 0);
             ok = mbar_wait_warp(&dq_full[it & 1], (it >> 1) & 1, ctl, kBSiteDqFull);
             if (!ok) break;
+            if (x == 0) SDPA_TR(4, it, 1);
             tc_fence_after();
             const uint32_t tDQ = tmem + lane_base + kColDP + (it & 1) * 64;
             uint32_t a0[32], a1[32];
@@ -375,8 +395,10 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive(&dq_empty[it & 1]);
+            if (x == 0) SDPA_TR(4, it, 2);
             if (x == 0) bulk_wait_read<0>();  // the previous step's reduce has finished reading the staging buffer
             named_bar_sync(2, 128);
+            if (x == 0) SDPA_TR(4, it, 3);
             if (x < D) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) sDQ[i * D + x] = __uint_as_float(a0[i]);
@@ -385,12 +407,14 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             fence_proxy_async_smem();
             named_bar_sync(2, 128);
+            if (x == 0) SDPA_TR(4, it, 4);
             if (x == 0) {
                 const int nq = min(64, L - q0);
                 float* dst = p.dq_acc + (static_cast<size_t>(h) * p.T + r0 + q0) * D;
                 bulk_reduce_add_f32(dst, sDQ, static_cast<uint32_t>(nq) * D * 4u);
                 bulk_commit();
             }
+            if (x == 0) SDPA_TR(4, it, 5);
         }
         if (x == 0) bulk_wait<0>();
     } else if (warp == 13) {
@@ -465,16 +489,20 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 uint32_t stage = 0, nstage = 1 % NS, nphase = (NS == 1) ? 1u : 0u;  // stage of step it / it+1
                 for (int it = 0; it < n_it && ok; ++it) {
                     const uint32_t buf = it & 1, ph = (it >> 1) & 1;
+                    SDPA_TR(1, it, 0);
                     if (it + 1 < n_it) {
                         ok = mbar_wait(&q_full[nstage], nphase, ctl, kBSiteQFull);
                         if (!ok) break;
+                        SDPA_TR(1, it, 1);
                         tc_fence_after();
                         issue_s(buf ^ 1, nstage);
                         umma_commit(&s_full[buf ^ 1]);
+                        SDPA_TR(1, it, 2);
                     }
                     // dV += P^T dO   (P^T from TMEM; the 64 queries of the step are the contraction index)
                     ok = mbar_wait(&p_ready[buf], ph, ctl, kBSitePReady);
                     if (!ok) break;
+                    SDPA_TR(1, it, 3);
                     tc_fence_after();
                     {
                         const uint64_t dod = do_mn_desc + stage * kStageStep;
@@ -485,6 +513,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                     idesc_acc, (it > 0 || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(&q_empty[stage]);
+                    SDPA_TR(1, it, 4);
                     stage = nstage;
                     if (++nstage == NS) { nstage = 0; nphase ^= 1; }
                 }
@@ -511,8 +540,10 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int it = 0; it < n_it && ok; ++it) {
                     const uint32_t buf = it & 1, ph = (it >> 1) & 1;
                     // dK += dS^T Q
+                    SDPA_TR(2, it, 0);
                     ok = mbar_wait(&ds_ready[buf], ph, ctl, kBSiteDsReady);
                     if (!ok) break;
+                    SDPA_TR(2, it, 1);
                     tc_fence_after();
                     {
                         const uint64_t dsd = ds_desc + buf * kDsStep;
@@ -524,6 +555,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                     umma_commit(&ds_free[buf]);
                     umma_commit(&q_empty[stage]);
+                    SDPA_TR(2, it, 2);
                     if (it + 1 < n_it) {
                         ok = mbar_wait(&q_full[nstage], nphase, ctl, kBSiteQFull);
                         if (!ok) break;
@@ -531,9 +563,11 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             ok = mbar_wait(&dq_empty[buf ^ 1], ph ^ ((it & 1) ? 0u : 1u), ctl, kBSiteDqEmpty);
                             if (!ok) break;
                         }
+                        SDPA_TR(2, it, 3);
                         tc_fence_after();
                         issue_dp(buf ^ 1, nstage);
                         umma_commit(&dp_full[buf ^ 1]);
+                        SDPA_TR(2, it, 4);
                     }
                     stage = nstage;
                     if (++nstage == NS) { nstage = 0; nphase ^= 1; }
@@ -544,8 +578,10 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const uint64_t ds_mn_desc = smem_desc_sw128(smem_u32(sDS), 0, 1024);                             // MN-major B
                 for (int it = 0; it < n_it && ok; ++it) {
                     const uint32_t buf = it & 1, ph = (it >> 1) & 1;
+                    SDPA_TR(3, it, 0);
                     ok = mbar_wait(&ds_ready[buf], ph, ctl, kBSiteDsReady);
                     if (!ok) break;
+                    SDPA_TR(3, it, 1);
                     tc_fence_after();
                     // dQ^T = K^T dS^T (overwrites the dP^T buffer of this step)
                     const uint64_t dsd = ds_mn_desc + buf * kDsStep;
@@ -556,6 +592,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                 idesc_dq, kk > 0);
                     umma_commit(&dq_full[buf]);
                     umma_commit(&ds_free[buf]);
+                    SDPA_TR(3, it, 2);
                 }
             }
             if (!ok) {

@@ -335,3 +335,9 @@ extern "C" const char* sdpa_status_string(int code) {
 }
 
 extern "C" int sdpa_last_cuda_error(void) { return tl_last_cuda_error; }
+
+#ifdef SDPA_TRACE
+extern "C" int sdpa_debug_trace(long long* host_out, int n) {
+    return static_cast<int>(cudaMemcpyFromSymbol(host_out, sdpa::g_trace, sizeof(long long) * n));
+}
+#endif
