@@ -66,7 +66,7 @@ struct BwdCfg {
     static constexpr int kSmemKV = 2 * kTileBytes;
     static constexpr int kSmemQdO = kQStages * kStageBytes;
     static constexpr int kSmemDS = 2 * 128 * 64 * 2;            // two dS^T buffers
-    static constexpr int kSmemRows = 2 * 2 * 64 * 4;            // lse / delta rows, double buffered
+    static constexpr int kSmemRows = kQStages * 2 * 64 * 4;     // lse / delta rows, one pair per Q/dO stage
     static constexpr int kSmemDQ = kStep * D * 4;               // fp32 staging of one dQ step for the bulk reduction
     static constexpr int kSmemBars = 256;
     // no alignment slack: the dynamic shared window is declared 1024-byte aligned and checked at run time
@@ -170,7 +170,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint8_t* sQdO = smem + Cfg::kSmemKV;  // stage s: Q step at s*kStageBytes, dO step right after it
     uint8_t* sDS = sQdO + Cfg::kSmemQdO;  // two buffers of [128 keys][64 queries] bf16, swizzled
     float* sDQ = reinterpret_cast<float*>(sDS + Cfg::kSmemDS);    // [64 queries][D] fp32
-    float* sRows = reinterpret_cast<float*>(sDS + Cfg::kSmemDS + Cfg::kSmemDQ);  // [2 buffers][lse2 | delta][64]
+    float* sRows = reinterpret_cast<float*>(sDS + Cfg::kSmemDS + Cfg::kSmemDQ);  // [NS stages][lse2 | delta][64]
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(sRows) + Cfg::kSmemRows);
     uint64_t* kv_full = bars;             // 1
     uint64_t* q_full = bars + 1;          // NS
@@ -195,14 +195,14 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         *abort_flag = 0;
         mbar_init(kv_full, 1);
         for (int i = 0; i < NS; ++i) {
-            mbar_init(&q_full[i], 1);
-            mbar_init(&q_empty[i], 2);  // released by the S^T/dV issuer and by the dP^T/dK issuer
+            mbar_init(&q_full[i], 33);  // TMA transaction arrival + 32 lanes that staged the lse / D_i rows
+            mbar_init(&q_empty[i], 3);  // one commit per MMA-issuing warp
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s_full[i], 1);
             mbar_init(&dp_full[i], 1);
-            mbar_init(&p_ready[i], 256);
-            mbar_init(&ds_ready[i], 256);
+            mbar_init(&p_ready[i], 128);
+            mbar_init(&ds_ready[i], 128);
             mbar_init(&ds_free[i], 2);  // dK issuer and dQ^T issuer
             mbar_init(&dq_full[i], 1);
             mbar_init(&dq_empty[i], 128);
@@ -228,124 +228,108 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // TMEM columns: S^T/P^T two buffers of 64, dP^T/dQ^T two buffers of 64, dV, dK
     constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
 
+    // Register re-balancing: one setmaxnreg instruction per warpgroup, executed by all of its warps.
+    if (warp < 8) setmaxnreg_inc<168>();
+    else setmaxnreg_dec<88>();
+
     if (warp < 8) {
-        // ------------------------------------------------------------ compute groups
-        const int wg = warp >> 2;          // owns query columns [32*wg, 32*wg + 32) of every step
+        // ------------------------------------------------------------ compute groups (ping-pong over steps)
+        // Group w owns the steps of parity w and the TMEM / dS buffers of index w, so one group's
+        // exponentials overlap the other group's dS and the MMAs of both.
+        const int wg = warp >> 2;
         const int r = tid & 127;           // key row inside the tile
         const int key = kv0 + r;           // key index inside the sequence
         const bool key_ok = key < L;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        const int row_which = tid >> 6, row_qi = tid & 63;  // threads 0..127 stage lse / delta rows
-        auto load_row = [&](int s) -> float {
-            float val = row_which == 0 ? INFINITY : 0.f;
-            if (tid < 128 && s < n_it) {
-                const int h = g * G + s / per_head;
-                const int qrow = (i_start + s % per_head) * 64 + row_qi;
-                if (qrow < L) {
-                    const size_t idx = static_cast<size_t>(h) * p.T + r0 + qrow;
-                    val = row_which == 0 ? p.lse[idx] * 1.4426950408889634f : p.delta[idx];
-                }
-            }
-            return val;
-        };
-        float pr[32];
+        const uint32_t tS = tmem + lane_base + kColS + wg * 64;
+        const uint32_t tDP = tmem + lane_base + kColDP + wg * 64;
+        uint8_t* ds_buf = sDS + wg * 16384;
         bool ok = true;
-        // A(s): P^T = exp2(S^T * scale_log2 - lse2) with masks; bf16 P^T overwrites the S^T columns
-        auto stage_a = [&](int s) -> bool {
-            if (tid == 0) SDPA_TR(0, s - 1, 4);
-            if (!mbar_wait_warp(&s_full[s & 1], (s >> 1) & 1, ctl, kBSiteSFull)) return false;
-            if (tid == 0) SDPA_TR(0, s - 1, 5);
-            tc_fence_after();
+        uint32_t stage = wg % NS, sphase = 0;
+        for (int s = wg; s < n_it && ok; s += 2) {
+            const uint32_t ph = (s >> 1) & 1;
             const int q0 = (i_start + s % per_head) * 64;
-            const uint32_t tS = tmem + lane_base + kColS + (s & 1) * 64 + wg * 32;
-            const float4* lse4 = reinterpret_cast<const float4*>(sRows + (s & 1) * 128 + wg * 32);
             const bool need_mask = (p.causal && q0 < kv0 + 128) || (kv0 + 128 > L);
-            uint32_t sr[32];
-            tmem_ld_x32(tS, sr);
-            tmem_wait_ld();
+            // rows (lse * log2e, D_i) of this step were staged by the producer warp together with Q / dO
+            if (r == 0) SDPA_TR(0, s, 0);
+            ok = mbar_wait_warp(&q_full[stage], sphase, ctl, kBSiteQFull);
+            if (!ok) break;
+            const float4* lse4 = reinterpret_cast<const float4*>(sRows + stage * 128);
+            const float4* dl4 = reinterpret_cast<const float4*>(sRows + stage * 128 + 64);
+            // A(s): P^T = exp2(S^T * scale_log2 - lse2) with masks; bf16 P^T overwrites the S^T columns
+            ok = mbar_wait_warp(&s_full[wg], ph, ctl, kBSiteSFull);
+            if (!ok) break;
+            if (r == 0) SDPA_TR(0, s, 1);
+            tc_fence_after();
+            float pr[64];
 #pragma unroll
-            for (int i4 = 0; i4 < 8; ++i4) {
-                const float4 l4 = lse4[i4];
-                const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+            for (int c = 0; c < 2; ++c) {
+                uint32_t sr[32];
+                tmem_ld_x32(tS + c * 32, sr);
+                tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int i = i4 * 4 + e;
-#ifdef SDPA_EXP_NO_EXP
-                    float v = fmaf(__uint_as_float(sr[i]), p.scale_log2, -lv[e]) * 1e-3f;
-#else
-                    float v = fast_exp2(fmaf(__uint_as_float(sr[i]), p.scale_log2, -lv[e]));
-#endif
-                    if (need_mask) {
-                        const int qq = q0 + wg * 32 + i;
-                        if (!key_ok || (p.causal && key > qq)) v = 0.f;
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    const float4 l4 = lse4[c * 8 + i4];
+                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = i4 * 4 + e;
+                        float v = fast_exp2(fmaf(__uint_as_float(sr[i]), p.scale_log2, -lv[e]));
+                        if (need_mask) {
+                            const int qq = q0 + c * 32 + i;
+                            if (!key_ok || (p.causal && key > qq)) v = 0.f;
+                        }
+                        pr[c * 32 + i] = v;
                     }
-                    pr[i] = v;
                 }
-            }
-            uint32_t pk[16];
+                uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
-            tmem_st_x16(tS, pk);
+                for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(pr[c * 32 + 2 * i], pr[c * 32 + 2 * i + 1]);
+                tmem_st_x16(tS + c * 16, pk);
+            }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&p_ready[s & 1]);
-            if (tid == 0) SDPA_TR(0, s - 1, 6);
-            return true;
-        };
-        // B(s): dS^T = P^T * (dP^T - D_i) -> bf16 -> swizzled shared memory
-        auto stage_b = [&](int s) -> bool {
-            if (tid == 0) SDPA_TR(0, s, 0);
-            if (!mbar_wait_warp(&dp_full[s & 1], (s >> 1) & 1, ctl, kBSiteDpFull)) return false;
-            if (tid == 0) SDPA_TR(0, s, 1);
+            mbar_arrive(&p_ready[wg]);
+            if (r == 0) SDPA_TR(0, s, 2);
+            // B(s): dS^T = P^T * (dP^T - D_i) -> bf16 -> swizzled shared memory
+            ok = mbar_wait_warp(&dp_full[wg], ph, ctl, kBSiteDpFull);
+            if (!ok) break;
+            if (r == 0) SDPA_TR(0, s, 3);
             tc_fence_after();
-            const uint32_t tDP = tmem + lane_base + kColDP + (s & 1) * 64 + wg * 32;
-            const float4* dl4 = reinterpret_cast<const float4*>(sRows + (s & 1) * 128 + 64 + wg * 32);
-            uint32_t dr[32];
-            tmem_ld_x32(tDP, dr);
-            tmem_wait_ld();
 #pragma unroll
-            for (int i4 = 0; i4 < 8; ++i4) {
-                const float4 d4 = dl4[i4];
-                pr[i4 * 4 + 0] *= (__uint_as_float(dr[i4 * 4 + 0]) - d4.x);
-                pr[i4 * 4 + 1] *= (__uint_as_float(dr[i4 * 4 + 1]) - d4.y);
-                pr[i4 * 4 + 2] *= (__uint_as_float(dr[i4 * 4 + 2]) - d4.z);
-                pr[i4 * 4 + 3] *= (__uint_as_float(dr[i4 * 4 + 3]) - d4.w);
+            for (int c = 0; c < 2; ++c) {
+                uint32_t dr[32];
+                tmem_ld_x32(tDP + c * 32, dr);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    const float4 d4 = dl4[c * 8 + i4];
+                    pr[c * 32 + i4 * 4 + 0] *= (__uint_as_float(dr[i4 * 4 + 0]) - d4.x);
+                    pr[c * 32 + i4 * 4 + 1] *= (__uint_as_float(dr[i4 * 4 + 1]) - d4.y);
+                    pr[c * 32 + i4 * 4 + 2] *= (__uint_as_float(dr[i4 * 4 + 2]) - d4.z);
+                    pr[c * 32 + i4 * 4 + 3] *= (__uint_as_float(dr[i4 * 4 + 3]) - d4.w);
+                }
             }
             if (s >= 2) {
-                if (!mbar_wait_warp(&ds_free[s & 1], ((s >> 1) - 1) & 1, ctl, kBSiteDsFree)) return false;
+                ok = mbar_wait_warp(&ds_free[wg], ph ^ 1, ctl, kBSiteDsFree);
+                if (!ok) break;
             }
-            if (tid == 0) SDPA_TR(0, s, 2);
-            uint8_t* ds_buf = sDS + (s & 1) * 16384;
+            if (r == 0) SDPA_TR(0, s, 4);
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int ch = 0; ch < 8; ++ch) {
                 uint4 w;
                 w.x = pack_bf16x2(pr[ch * 8 + 0], pr[ch * 8 + 1]);
                 w.y = pack_bf16x2(pr[ch * 8 + 2], pr[ch * 8 + 3]);
                 w.z = pack_bf16x2(pr[ch * 8 + 4], pr[ch * 8 + 5]);
                 w.w = pack_bf16x2(pr[ch * 8 + 6], pr[ch * 8 + 7]);
-                *reinterpret_cast<uint4*>(ds_buf + sw128_offset(r, wg * 4 + ch)) = w;
+                *reinterpret_cast<uint4*>(ds_buf + sw128_offset(r, ch)) = w;
             }
             fence_proxy_async_smem();
             tc_fence_before();
-            mbar_arrive(&ds_ready[s & 1]);
-            if (tid == 0) SDPA_TR(0, s, 3);
-            return true;
-        };
-
-        float pre = load_row(0);
-        if (tid < 128) sRows[row_which * 64 + row_qi] = pre;
-        pre = load_row(1);
-        named_bar_sync(1, 256);
-        ok = stage_a(0);
-        for (int it = 0; it < n_it && ok; ++it) {
-            ok = stage_b(it);
-            if (!ok) break;
-            if (it + 1 < n_it) {
-                if (tid < 128) sRows[((it + 1) & 1) * 128 + row_which * 64 + row_qi] = pre;
-                pre = load_row(it + 2);
-                named_bar_sync(1, 256);
-                ok = stage_a(it + 1);
-            }
+            mbar_arrive(&ds_ready[wg]);
+            if (r == 0) SDPA_TR(0, s, 5);
+            stage += 2;
+            if (stage >= NS) { stage -= NS; sphase ^= 1; }
         }
         if (ok) ok = mbar_wait_warp(dkv_full, 0, ctl, kBSiteDkvFull);
         if (ok) {
@@ -396,44 +380,57 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tc_fence_before();
             mbar_arrive(&dq_empty[it & 1]);
             if (x == 0) SDPA_TR(4, it, 2);
-            if (x == 0) bulk_wait_read<0>();  // the previous step's reduce has finished reading the staging buffer
-            named_bar_sync(2, 128);
-            if (x == 0) SDPA_TR(4, it, 3);
-            if (x < D) {
+            // Two halves of 32 query rows, each its own bulk group: the rows of one half are rewritten
+            // while the bulk engine is still reading the other half of the previous step.
+            const int nq = min(64, L - q0);
+            float* dst = p.dq_acc + (static_cast<size_t>(h) * p.T + r0 + q0) * D;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) sDQ[i * D + x] = __uint_as_float(a0[i]);
+            for (int hf = 0; hf < 2; ++hf) {
+                if (x == 0) bulk_wait_read<1>();  // the group that last read this half has finished reading
+                named_bar_sync(2, 128);
+                if (x < D) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) sDQ[(32 + i) * D + x] = __uint_as_float(a1[i]);
+                    for (int i = 0; i < 32; ++i)
+                        sDQ[(hf * 32 + i) * D + x] = __uint_as_float(hf == 0 ? a0[i] : a1[i]);
+                }
+                fence_proxy_async_smem();
+                named_bar_sync(2, 128);
+                if (x == 0) {
+                    const int rows = min(32, nq - hf * 32);
+#ifndef SDPA_EXP_NO_REDUCE
+                    if (rows > 0)
+                        bulk_reduce_add_f32(dst + hf * 32 * D, sDQ + hf * 32 * D, static_cast<uint32_t>(rows) * D * 4u);
+#endif
+                    bulk_commit();  // committed even when empty, so the group count per step is fixed
+                }
+                if (x == 0 && hf == 0) SDPA_TR(4, it, 3);
             }
-            fence_proxy_async_smem();
-            named_bar_sync(2, 128);
             if (x == 0) SDPA_TR(4, it, 4);
-            if (x == 0) {
-                const int nq = min(64, L - q0);
-                float* dst = p.dq_acc + (static_cast<size_t>(h) * p.T + r0 + q0) * D;
-                bulk_reduce_add_f32(dst, sDQ, static_cast<uint32_t>(nq) * D * 4u);
-                bulk_commit();
-            }
             if (x == 0) SDPA_TR(4, it, 5);
         }
         if (x == 0) bulk_wait<0>();
     } else if (warp == 13) {
-        // ------------------------------------------------------------ TMA producer
-        if (elect_one()) {
+        // ------------------------------------------------------------ producer warp (all 32 lanes)
+        // Lane 0 issues the TMA loads; every lane stages two (lse * log2e, D_i) pairs of the step's 64
+        // query rows in shared memory.  q_full collects the TMA bytes and the 32 lane arrivals.
+        const int lane = tid & 31;
+        if (lane == 0) {
             mbar_arrive_expect_tx(kv_full, 2 * Cfg::kTileBytes);
 #pragma unroll
             for (int a = 0; a < D / 64; ++a) {
                 tma_load_3d(sK + a * Cfg::kAtomBytes, &map_k, kv_full, a * 64, g, r0 + kv0);
                 tma_load_3d(sV + a * Cfg::kAtomBytes, &map_v, kv_full, a * 64, g, r0 + kv0);
             }
-            bool ok = true;
-            int it = 0;
-            for (; it < n_it && ok; ++it) {
-                const int st = it % NS;
-                ok = mbar_wait(&q_empty[st], ((it / NS) & 1) ^ 1, ctl, kBSiteQEmpty);
-                if (!ok) break;
-                const int h = g * G + it / per_head;
-                const int q0 = (i_start + it % per_head) * 64;
+        }
+        bool ok = true;
+        int it = 0;
+        uint32_t st = 0, ph = 0;
+        for (; it < n_it && ok; ++it) {
+            ok = mbar_wait_warp(&q_empty[st], ph ^ 1, ctl, kBSiteQEmpty);
+            if (!ok) break;
+            const int h = g * G + it / per_head;
+            const int q0 = (i_start + it % per_head) * 64;
+            if (lane == 0) {
                 uint8_t* dst = sQdO + st * Cfg::kStageBytes;
                 mbar_arrive_expect_tx(&q_full[st], Cfg::kStageBytes);
 #pragma unroll
@@ -443,26 +440,39 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                 r0 + q0);
                 }
             }
-            if (!ok) {
-                mbar_wait(kv_full, 0, ctl, kBSiteDrain);
-                for (int back = 1; back <= NS && back <= it; ++back) {
-                    const int i2 = it - back;
-                    mbar_wait(&q_full[i2 % NS], (i2 / NS) & 1, ctl, kBSiteDrain);
+            float* rows = sRows + st * 128;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int qi = lane * 2 + e;
+                float lv = INFINITY, dv = 0.f;  // rows past the sequence end: P = exp2(-inf) = 0
+                if (q0 + qi < L) {
+                    const size_t idx = static_cast<size_t>(h) * p.T + r0 + q0 + qi;
+                    lv = p.lse[idx] * 1.4426950408889634f;
+                    dv = p.delta[idx];
                 }
+                rows[qi] = lv;
+                rows[64 + qi] = dv;
+            }
+            mbar_arrive(&q_full[st]);
+            if (++st == NS) { st = 0; ph ^= 1; }
+        }
+        if (!ok && lane == 0) {
+            mbar_wait(kv_full, 0, ctl, kBSiteDrain);
+            for (int back = 1; back <= NS && back <= it; ++back) {
+                const int i2 = it - back;
+                mbar_wait(&q_full[i2 % NS], (i2 / NS) & 1, ctl, kBSiteDrain);
             }
         }
-    } else if (warp == 12 || warp == 14 || warp == 15) {
-        // ------------------------------------------------------------ MMA issuers
-        // One thread can start a tcgen05.mma only about every 90-100 cycles, so the MMAs of a step are
-        // spread over three issuing warps:  warp 12: S^T(i+1), dV(i);  warp 14: dK(i), dP^T(i+1);
-        // warp 15: dQ^T(i).  Hazards between warps are all covered by mbarriers (see the header).
+    } else {
+        // ------------------------------------------------------------ MMA issuers (warps 12, 14, 15)
+        // The issuing thread's own instruction stream bounds its MMA rate, so the MMAs of a step are
+        // spread over three warps:  warp 12: dV(i), S^T(i+2);  warp 14: dK(i);
+        // warp 15: dQ^T(i), then (after the reduction group drained it) dP^T(i+2) into the same columns.
         if (elect_one()) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, false, false);   // S^T, dP^T: keys x 64 queries
             constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);   // dV, dK: keys x d
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, 64, true, true);    // dQ^T: d x 64 queries
             constexpr uint32_t kLboK = (D == 128) ? Cfg::kAtomBytes : 0;           // D=64: rows 64..127 repeat, unused
-            // Descriptors are built once; inside the loops they only advance by constants, because
-            // every extra instruction of the issuing thread delays the next tcgen05.mma by several cycles.
             constexpr uint64_t kStageStep = Cfg::kStageBytes >> 4;
             constexpr uint64_t kDsStep = 16384 >> 4;
             auto kmaj = [](int kk, int atom_bytes) -> uint64_t {
@@ -480,63 +490,51 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     for (int kk = 0; kk < Cfg::kKSteps; ++kk)
                         umma_ss(d, k_desc + kmaj(kk, Cfg::kAtomBytes), qd + kmaj(kk, Cfg::kStepAtomBytes), idesc_s, kk > 0);
                 };
-                if (ok) ok = mbar_wait(&q_full[0], 0, ctl, kBSiteQFull);
-                if (ok) {
+                // prologue: S^T(0), S^T(1)
+                for (int s = 0; s < 2 && s < n_it && ok; ++s) {
+                    ok = mbar_wait(&q_full[s % NS], 0, ctl, kBSiteQFull);
+                    if (!ok) break;
                     tc_fence_after();
-                    issue_s(0, 0);
-                    umma_commit(&s_full[0]);
+                    issue_s(s, s % NS);
+                    umma_commit(&s_full[s]);
                 }
-                uint32_t stage = 0, nstage = 1 % NS, nphase = (NS == 1) ? 1u : 0u;  // stage of step it / it+1
+                uint32_t stage = 0;                        // stage of step it
+                uint32_t stage2 = 2 % NS, phase2 = (2 >= NS) ? 1u : 0u;  // stage / phase of step it+2
                 for (int it = 0; it < n_it && ok; ++it) {
                     const uint32_t buf = it & 1, ph = (it >> 1) & 1;
                     SDPA_TR(1, it, 0);
-                    if (it + 1 < n_it) {
-                        ok = mbar_wait(&q_full[nstage], nphase, ctl, kBSiteQFull);
-                        if (!ok) break;
-                        SDPA_TR(1, it, 1);
-                        tc_fence_after();
-                        issue_s(buf ^ 1, nstage);
-                        umma_commit(&s_full[buf ^ 1]);
-                        SDPA_TR(1, it, 2);
-                    }
                     // dV += P^T dO   (P^T from TMEM; the 64 queries of the step are the contraction index)
                     ok = mbar_wait(&p_ready[buf], ph, ctl, kBSitePReady);
                     if (!ok) break;
-                    SDPA_TR(1, it, 3);
+                    SDPA_TR(1, it, 1);
                     tc_fence_after();
                     {
                         const uint64_t dod = do_mn_desc + stage * kStageStep;
                         const uint32_t a = tmem + kColS + buf * 64;
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
-                            umma_ts(tmem + kColDV, a + (kk >> 1) * 32 + (kk & 1) * 8, dod + static_cast<uint64_t>(kk * (2048 >> 4)),
-                                    idesc_acc, (it > 0 || kk > 0) ? 1u : 0u);
+                            umma_ts(tmem + kColDV, a + kk * 8, dod + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_acc,
+                                    (it > 0 || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(&q_empty[stage]);
-                    SDPA_TR(1, it, 4);
-                    stage = nstage;
-                    if (++nstage == NS) { nstage = 0; nphase ^= 1; }
+                    SDPA_TR(1, it, 2);
+                    if (it + 2 < n_it) {  // S^T(it+2) overwrites P^T(it): same thread, issued in order after dV(it)
+                        ok = mbar_wait(&q_full[stage2], phase2, ctl, kBSiteQFull);
+                        if (!ok) break;
+                        SDPA_TR(1, it, 3);
+                        tc_fence_after();
+                        issue_s(buf, stage2);
+                        umma_commit(&s_full[buf]);
+                        SDPA_TR(1, it, 4);
+                    }
+                    if (++stage == NS) stage = 0;
+                    if (++stage2 == NS) { stage2 = 0; phase2 ^= 1; }
                 }
                 if (ok) umma_commit(dkv_full);
             } else if (warp == 14) {
-                const uint64_t v_desc = smem_desc_sw128(smem_u32(sV), 0, 1024);
-                const uint64_t do_desc = smem_desc_sw128(smem_u32(sQdO) + Cfg::kStepBytes, 0, 1024);            // K-major B
                 const uint64_t q_mn_desc = smem_desc_sw128(smem_u32(sQdO), Cfg::kStepAtomBytes, 1024);           // MN-major B
                 const uint64_t ds_desc = smem_desc_sw128(smem_u32(sDS), 0, 1024);                                // K-major A
-                auto issue_dp = [&](uint32_t buf, uint32_t stage) {  // dP^T = V dO^T into dP buffer `buf`
-                    const uint64_t dd = do_desc + stage * kStageStep;
-                    const uint32_t d = tmem + kColDP + buf * 64;
-#pragma unroll
-                    for (int kk = 0; kk < Cfg::kKSteps; ++kk)
-                        umma_ss(d, v_desc + kmaj(kk, Cfg::kAtomBytes), dd + kmaj(kk, Cfg::kStepAtomBytes), idesc_s, kk > 0);
-                };
-                if (ok) ok = mbar_wait(&q_full[0], 0, ctl, kBSiteQFull);
-                if (ok) {
-                    tc_fence_after();
-                    issue_dp(0, 0);
-                    umma_commit(&dp_full[0]);
-                }
-                uint32_t stage = 0, nstage = 1 % NS, nphase = (NS == 1) ? 1u : 0u;
+                uint32_t stage = 0;
                 for (int it = 0; it < n_it && ok; ++it) {
                     const uint32_t buf = it & 1, ph = (it >> 1) & 1;
                     // dK += dS^T Q
@@ -545,54 +543,81 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     if (!ok) break;
                     SDPA_TR(2, it, 1);
                     tc_fence_after();
-                    {
-                        const uint64_t dsd = ds_desc + buf * kDsStep;
-                        const uint64_t qd = q_mn_desc + stage * kStageStep;
+                    const uint64_t dsd = ds_desc + buf * kDsStep;
+                    const uint64_t qd = q_mn_desc + stage * kStageStep;
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            umma_ss(tmem + kColDK, dsd + static_cast<uint64_t>(kk * 2), qd + static_cast<uint64_t>(kk * (2048 >> 4)),
-                                    idesc_acc, (it > 0 || kk > 0) ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_ss(tmem + kColDK, dsd + static_cast<uint64_t>(kk * 2), qd + static_cast<uint64_t>(kk * (2048 >> 4)),
+                                idesc_acc, (it > 0 || kk > 0) ? 1u : 0u);
                     umma_commit(&ds_free[buf]);
                     umma_commit(&q_empty[stage]);
                     SDPA_TR(2, it, 2);
-                    if (it + 1 < n_it) {
-                        ok = mbar_wait(&q_full[nstage], nphase, ctl, kBSiteQFull);
-                        if (!ok) break;
-                        if (it >= 1) {  // the dQ^T that lived in this buffer has been drained
-                            ok = mbar_wait(&dq_empty[buf ^ 1], ph ^ ((it & 1) ? 0u : 1u), ctl, kBSiteDqEmpty);
-                            if (!ok) break;
-                        }
-                        SDPA_TR(2, it, 3);
-                        tc_fence_after();
-                        issue_dp(buf ^ 1, nstage);
-                        umma_commit(&dp_full[buf ^ 1]);
-                        SDPA_TR(2, it, 4);
-                    }
-                    stage = nstage;
-                    if (++nstage == NS) { nstage = 0; nphase ^= 1; }
+                    if (++stage == NS) stage = 0;
                 }
                 if (ok) umma_commit(dkv_full);
             } else {
                 const uint64_t kt_desc = smem_desc_sw128(smem_u32(sK), kLboK, 1024);                             // MN-major A
                 const uint64_t ds_mn_desc = smem_desc_sw128(smem_u32(sDS), 0, 1024);                             // MN-major B
-                for (int it = 0; it < n_it && ok; ++it) {
-                    const uint32_t buf = it & 1, ph = (it >> 1) & 1;
-                    SDPA_TR(3, it, 0);
-                    ok = mbar_wait(&ds_ready[buf], ph, ctl, kBSiteDsReady);
-                    if (!ok) break;
-                    SDPA_TR(3, it, 1);
-                    tc_fence_after();
-                    // dQ^T = K^T dS^T (overwrites the dP^T buffer of this step)
-                    const uint64_t dsd = ds_mn_desc + buf * kDsStep;
+                const uint64_t v_desc = smem_desc_sw128(smem_u32(sV), 0, 1024);
+                const uint64_t do_desc = smem_desc_sw128(smem_u32(sQdO) + Cfg::kStepBytes, 0, 1024);            // K-major B
+                auto issue_dp = [&](uint32_t buf, uint32_t stage) {  // dP^T = V dO^T into dP buffer `buf`
+                    const uint64_t dd = do_desc + stage * kStageStep;
                     const uint32_t d = tmem + kColDP + buf * 64;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        umma_ss(d, kt_desc + static_cast<uint64_t>(kk * (2048 >> 4)), dsd + static_cast<uint64_t>(kk * (2048 >> 4)),
-                                idesc_dq, kk > 0);
-                    umma_commit(&dq_full[buf]);
-                    umma_commit(&ds_free[buf]);
-                    SDPA_TR(3, it, 2);
+                    for (int kk = 0; kk < Cfg::kKSteps; ++kk)
+                        umma_ss(d, v_desc + kmaj(kk, Cfg::kAtomBytes), dd + kmaj(kk, Cfg::kStepAtomBytes), idesc_s, kk > 0);
+                };
+                // Event loop: issue whichever of dP^T(np) / dQ^T(nq) has its inputs ready, so that waiting
+                // for the reduction group to drain one buffer never delays the other buffer's dQ^T.
+                int nq = 0, np = 0;
+                uint32_t stage_p = 0, phase_p = 0;  // Q/dO stage and phase of step np
+                long long t_idle = 0;
+                bool idle = false;
+                while (ok && (nq < n_it || np < n_it)) {
+                    bool did = false;
+                    if (np < n_it && np < nq + 2) {
+                        // dP^T(np) reuses the columns of dQ^T(np-2): wait until the reduction group has read it
+                        if (mbar_try_wait(&q_full[stage_p], phase_p) &&
+                            (np < 2 || mbar_try_wait(&dq_empty[np & 1], ((np >> 1) - 1) & 1))) {
+                            SDPA_TR(3, np, 3);
+                            tc_fence_after();
+                            issue_dp(np & 1, stage_p);
+                            umma_commit(&dp_full[np & 1]);
+                            umma_commit(&q_empty[stage_p]);
+                            SDPA_TR(3, np, 4);
+                            ++np;
+                            if (++stage_p == NS) { stage_p = 0; phase_p ^= 1; }
+                            did = true;
+                        }
+                    }
+                    if (!did && nq < n_it && mbar_try_wait(&ds_ready[nq & 1], (nq >> 1) & 1)) {
+                        SDPA_TR(3, nq, 1);
+                        tc_fence_after();
+                        // dQ^T = K^T dS^T (overwrites the dP^T buffer of this step)
+                        const uint64_t dsd = ds_mn_desc + (nq & 1) * kDsStep;
+                        const uint32_t d = tmem + kColDP + (nq & 1) * 64;
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            umma_ss(d, kt_desc + static_cast<uint64_t>(kk * (2048 >> 4)), dsd + static_cast<uint64_t>(kk * (2048 >> 4)),
+                                    idesc_dq, kk > 0);
+                        umma_commit(&dq_full[nq & 1]);
+                        umma_commit(&ds_free[nq & 1]);
+                        SDPA_TR(3, nq, 2);
+                        ++nq;
+                        did = true;
+                    }
+                    if (did) {
+                        idle = false;
+                    } else if (!idle) {
+                        idle = true;
+                        t_idle = clock64();
+                    } else if (*ctl.abort) {
+                        ok = false;
+                    } else if (clock64() - t_idle > SDPA_WAIT_LIMIT_CYCLES) {
+                        *ctl.abort = 1;
+                        atomicCAS(ctl.g_status, 0, (kBSiteDqEmpty << 8) | kStatusTimeout);
+                        ok = false;
+                    }
                 }
             }
             if (!ok) {
