@@ -51,6 +51,7 @@ extern "C" {
 #define SDPA_ERR_WORKSPACE (-4) /* workspace missing, misaligned or too small */
 #define SDPA_ERR_ARCH (-5)      /* current device is not compute capability 10.x */
 #define SDPA_ERR_CUDA (-6)      /* a CUDA runtime/driver call failed; see sdpa_last_cuda_error */
+#define SDPA_ERR_STATIC_SCRATCH (-7) /* problem needs more than SDPA_STATIC_SCRATCH_BYTES of built-in scratch */
 
 #define SDPA_STATUS_TIMEOUT 1        /* a device-side wait gave up; outputs of that call are invalid */
 #define SDPA_STATUS_BAD_CU_SEQLENS 2 /* cu_seqlens contradicts total_tokens / max_seqlen */
@@ -92,6 +93,41 @@ int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B,
              int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Backward pass for callers that may not allocate device memory (the paper has no counterpart: this
+ * is a convenience of this library, not one of its operators).
+ *
+ * sdpa_bwd needs scratch (the fp32 dQ accumulator and the D_i rows) that the caller normally
+ * allocates.  Some callers cannot: a plug-in living inside a host runtime that hands out a fixed
+ * arena at start-up and forbids cudaMalloc afterwards, a latency-critical loop in which the implicit
+ * device synchronisation of an allocation is unacceptable, or code under a no-dynamic-allocation
+ * rule after initialisation.  For them this entry point computes exactly what sdpa_bwd computes, with
+ * the same arguments minus the workspace, and takes its scratch from a fixed array of
+ * SDPA_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library image: every GPU on which the
+ * library is used holds these 32 MiB from the moment the library's module is loaded on it until the
+ * process exits.  The call itself allocates and frees nothing (no cudaMalloc / cudaFree, no
+ * allocating library routine); inputs and outputs are still caller-owned device buffers.
+ *
+ *  - Limit: sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen) must not exceed
+ *    SDPA_STATIC_SCRATCH_BYTES (about total_tokens * Hq * (D + 1) * 4 bytes; e.g. T*Hq <= 65,000
+ *    at D = 128).  Larger problems are rejected with SDPA_ERR_STATIC_SCRATCH before anything is
+ *    launched; use sdpa_bwd with your own workspace for those.
+ *  - First use on a device: the first call made while a given device is current looks up the
+ *    device address of the array (cudaGetSymbolAddress, once per device) before launching.  Make that
+ *    first call during start-up, before any stream capture is begun on that device.
+ *  - The array is shared by every call in the process and keeps whatever the previous call left in
+ *    it.  Each call clears the part it accumulates into before using it, so calls that run one after
+ *    the other on the GPU are independent; two calls that overlap on the GPU (different streams, or
+ *    different host threads on different streams) race on the array and corrupt each other's dq.
+ *    Serialise them, or give the concurrent ones sdpa_bwd with separate workspaces.
+ * Errors and status reporting are those of sdpa_bwd.
+ */
+#define SDPA_STATIC_SCRATCH_BYTES (32u << 20)
+int sdpa_bwd_static_scratch(const void* q, const void* k, const void* v, const void* o,
+                            const float* lse, const void* dout, void* dq, void* dk, void* dv,
+                            const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D, int causal,
+                            float scale, int total_tokens, int max_seqlen, void* stream);
 
 /*
  * Whole step with HOST buffers (no counterpart in the paper's operator list beyond composing the

@@ -18,7 +18,7 @@ _LIB = None
 SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
-           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events")
+           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch")
 
 
 class SdpaError(RuntimeError):
@@ -47,6 +47,8 @@ def load():
     lib.sdpa_fwd_bwd_host.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp, ctypes.c_size_t, vp]
     lib.sdpa_bwd_profile_events.restype = ci
     lib.sdpa_bwd_profile_events.argtypes = [vp, vp]
+    lib.sdpa_bwd_static_scratch.restype = ci
+    lib.sdpa_bwd_static_scratch.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp]
     lib.sdpa_query_status.restype = ci
     lib.sdpa_query_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.sdpa_status_string.restype = ctypes.c_char_p
@@ -126,6 +128,29 @@ def sdpa_bwd(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, s
                       _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
     _check(rc, "sdpa_bwd")
     return dq, dk, dv
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+SDPA_ERR_STATIC_SCRATCH = -7
+
+
+def sdpa_bwd_static_scratch(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, scale: float,
+                            dq, dk, dv, stream=None):
+    """sdpa_bwd without a workspace argument, for callers that must not allocate device memory:
+    the scratch is a fixed 32 MiB array inside the library (see include/sdpa.h for the size limit,
+    the first-call set-up and the rule that overlapping calls race on it).  The outputs dq, dk, dv
+    are required, because this wrapper allocates nothing either.  Returns the library's return code
+    instead of raising when the problem is too large for the built-in scratch."""
+    lib = load()
+    T, Hq, Hkv, D = _dims(q, k)
+    B = cu_seqlens.numel() - 1
+    rc = lib.sdpa_bwd_static_scratch(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk),
+                                     _ptr(dv), _ptr(cu_seqlens), B, Hq, Hkv, D, int(bool(causal)), float(scale), T,
+                                     int(max_seqlen), _stream_ptr(stream))
+    if rc == SDPA_ERR_STATIC_SCRATCH:
+        return rc
+    _check(rc, "sdpa_bwd_static_scratch")
+    return rc
 
 
 def sdpa_host_staging_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen) -> int:

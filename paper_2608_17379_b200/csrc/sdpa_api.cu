@@ -249,6 +249,50 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
     return SDPA_OK;
 }
 
+// ------------------------------------------------------------------ built-in scratch (no allocation)
+// Scratch for sdpa_bwd_static_scratch.  It lives in the library image, so a GPU that loads the
+// library keeps these bytes until the process ends.
+static __device__ __align__(256) unsigned char g_static_scratch[SDPA_STATIC_SCRATCH_BYTES];
+// In host code the name g_static_scratch only stands for the symbol; it is not an address the GPU
+// can use.  The real device address differs per device and is looked up once per device below.
+static void* g_static_scratch_addr[sdpa::kMaxDevices];
+
+static int static_scratch_address(void** out) {
+    int dev = -1;
+    SDPA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= sdpa::kMaxDevices) return SDPA_ERR_ARCH;
+    std::lock_guard<std::mutex> lock(sdpa::g_mutex);
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* addr = nullptr;
+        SDPA_CUDA_TRY(cudaGetSymbolAddress(&addr, g_static_scratch));  // for the device that is current now
+        if (addr == nullptr) {
+            sdpa::tl_last_cuda_error = static_cast<int>(cudaErrorInvalidSymbol);
+            return SDPA_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = addr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return SDPA_OK;
+}
+
+extern "C" int sdpa_bwd_static_scratch(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                                       const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens,
+                                       int B, int Hq, int Hkv, int D, int causal, float scale, int total_tokens,
+                                       int max_seqlen, void* stream) {
+    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen);
+    if (rc != SDPA_OK) return rc;
+    if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
+    const size_t need = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
+    if (need == 0 || need > static_cast<size_t>(SDPA_STATIC_SCRATCH_BYTES)) return SDPA_ERR_STATIC_SCRATCH;
+    void* scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != SDPA_OK) return rc;
+    // sdpa_bwd clears the dQ accumulator inside the scratch before it accumulates into it and
+    // overwrites the D_i rows, so nothing of an earlier call survives into this one.
+    return sdpa_bwd(q, k, v, o, lse, dout, dq, dk, dv, cu_seqlens, B, Hq, Hkv, D, causal, scale, total_tokens,
+                    max_seqlen, scratch, static_cast<size_t>(SDPA_STATIC_SCRATCH_BYTES), stream);
+}
+
 extern "C" int sdpa_bwd_profile_events(void* ev_main_start, void* ev_main_stop) {
     tl_ev_main_start = static_cast<cudaEvent_t>(ev_main_start);
     tl_ev_main_stop = static_cast<cudaEvent_t>(ev_main_stop);
@@ -327,6 +371,8 @@ extern "C" const char* sdpa_status_string(int code) {
         case SDPA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case SDPA_ERR_ARCH: return "device is not compute capability 10.x";
         case SDPA_ERR_CUDA: return "CUDA runtime or driver call failed";
+        case SDPA_ERR_STATIC_SCRATCH:
+            return "problem exceeds the built-in scratch (SDPA_STATIC_SCRATCH_BYTES); use sdpa_bwd with a workspace";
         case SDPA_STATUS_TIMEOUT: return "device-side wait timed out";
         case SDPA_STATUS_BAD_CU_SEQLENS: return "cu_seqlens inconsistent with total_tokens/max_seqlen";
         case SDPA_STATUS_INTERNAL: return "kernel launch precondition violated";
