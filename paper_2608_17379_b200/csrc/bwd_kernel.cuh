@@ -577,8 +577,8 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     bool did = false;
                     if (np < n_it && np < nq + 2) {
                         // dP^T(np) reuses the columns of dQ^T(np-2): wait until the reduction group has read it
-                        if (mbar_try_wait(&q_full[stage_p], phase_p) &&
-                            (np < 2 || mbar_try_wait(&dq_empty[np & 1], ((np >> 1) - 1) & 1))) {
+                        if (mbar_test_wait(&q_full[stage_p], phase_p) &&
+                            (np < 2 || mbar_test_wait(&dq_empty[np & 1], ((np >> 1) - 1) & 1))) {
                             SDPA_TR(3, np, 3);
                             tc_fence_after();
                             issue_dp(np & 1, stage_p);
@@ -590,7 +590,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             did = true;
                         }
                     }
-                    if (!did && nq < n_it && mbar_try_wait(&ds_ready[nq & 1], (nq >> 1) & 1)) {
+                    if (!did && nq < n_it && mbar_test_wait(&ds_ready[nq & 1], (nq >> 1) & 1)) {
                         SDPA_TR(3, nq, 1);
                         tc_fence_after();
                         // dQ^T = K^T dS^T (overwrites the dP^T buffer of this step)
