@@ -30,6 +30,9 @@ from paper_2608_17379_b200 import workloads as W  # noqa: E402
 
 METRIC = "SDPA fwd+bwd TFLOPS (bf16, device-timed)"
 NOMINAL_BF16_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this same command on
+# the c3 workload (profiles/sdpa_kernels_c3_dram.md); null for other workloads.
+NCU_DRAM_TRAFFIC_C3 = {"sdpa_bwd_kernel<128>": 639476992 + 302121984, "sdpa_fwd_kernel<128>": 100827904 + 32541184}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -312,9 +315,12 @@ def main():
                 "frac_of_nominal_2250": bwd_tf / NOMINAL_BF16_TFLOPS, "kernels": 3},
         "roofline": {"bound": "tensor", "kernel": "sdpa_bwd_kernel<128>", "achieved": main_tf, "peak": peak,
                      "unit": "TFLOP/s", "frac": main_tf / peak, "peak_source": f"{peaks['_source']} bf16 burst",
-                     "ms_per_launch": main_med, "flops_per_launch": w.bwd_flops(), "traffic": None,
+                     "ms_per_launch": main_med, "flops_per_launch": w.bwd_flops(),
+                     "traffic": NCU_DRAM_TRAFFIC_C3["sdpa_bwd_kernel<128>"] if w.name == "c3" else None,
+                     "traffic_unit": "bytes per launch (ncu dram read+write)",
                      "fwd_kernel": {"kernel": "sdpa_fwd_kernel<128>", "achieved": fwd_tf, "frac": fwd_tf / peak,
-                                    "ms_per_launch": fwd_ms, "flops_per_launch": w.fwd_flops()},
+                                    "ms_per_launch": fwd_ms, "flops_per_launch": w.fwd_flops(),
+                                    "traffic": NCU_DRAM_TRAFFIC_C3["sdpa_fwd_kernel<128>"] if w.name == "c3" else None},
                      "hbm_min_bytes_per_step": w.min_bytes_fwd() + w.min_bytes_bwd(),
                      "hbm_gbs_at_min_bytes": (w.min_bytes_fwd() + w.min_bytes_bwd()) / (step_ms * 1e-3) / 1e9,
                      "hbm_peak_gbs": float(peaks["hbm_gbs"])},
