@@ -102,6 +102,20 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity when not distributed)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def whole_job_tflops(flops_per_rank: float, world: int, ms: float) -> float:
+    """Aggregate throughput of `world` replicas that each did `flops_per_rank` in `ms` (max over ranks)."""
+    return world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 def oracle_sample(w: W.Workload, inputs_bits, budget_s: float):
     """Time the fp64 oracle (fwd+bwd) on whole (sequence, kv-head) slices of the workload until
     about `budget_s` seconds of CPU work are done.  Returns (flops_done, seconds, n_slices, threads)."""
@@ -250,10 +264,7 @@ def main():
     fwd_ms = float(np.median([e_f0[i].elapsed_time(e_f1[i]) for i in range(K)]))
     bwd_ms = float(np.median([e_f1[i].elapsed_time(e_b1[i]) for i in range(K)]))
     step_ms = total_ms / K
-    if dist is not None:
-        t = torch.tensor([step_ms, fwd_ms, bwd_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms, fwd_ms, bwd_ms = (float(x) for x in t.tolist())
+    step_ms, fwd_ms, bwd_ms = max_over_ranks([step_ms, fwd_ms, bwd_ms], dist, "cuda")
 
     # ---- end to end through the C ABI with HOST buffers (copies inside the timed region)
     o_h = torch.empty((T, Hq, D), dtype=torch.bfloat16).pin_memory()
@@ -278,10 +289,7 @@ def main():
     s1.record()
     barrier()
     e2e_ms = s0.elapsed_time(s1) / Ke
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    (e2e_ms,) = max_over_ranks([e2e_ms], dist, "cuda")
     assert binding.query_status() == (0, 0)
     h2d = 2 * (T * Hq * D * 2) + 2 * (T * Hkv * D * 2) + (w.B + 1) * 4
     d2h = 2 * (T * Hq * D * 2) + 2 * (T * Hkv * D * 2) + T * Hq * 4
@@ -293,7 +301,7 @@ def main():
 
     peaks = measured_peaks()
     step_flops = w.fwd_flops() + w.bwd_flops()
-    value = world * step_flops / (step_ms * 1e-3) / 1e12
+    value = whole_job_tflops(step_flops, world, step_ms)
     fwd_tf = w.fwd_flops() / (fwd_ms * 1e-3) / 1e12
     bwd_tf = w.bwd_flops() / (bwd_ms * 1e-3) / 1e12
     main_med = float(np.median(main_ms))
@@ -324,7 +332,7 @@ def main():
                      "hbm_min_bytes_per_step": w.min_bytes_fwd() + w.min_bytes_bwd(),
                      "hbm_gbs_at_min_bytes": (w.min_bytes_fwd() + w.min_bytes_bwd()) / (step_ms * 1e-3) / 1e9,
                      "hbm_peak_gbs": float(peaks["hbm_gbs"])},
-        "e2e": {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_tflops(step_flops, world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "sdpa_fwd_bwd_host (pinned host buffers)"},
         "gpu_launches": 4 * K,
         "clocks": clocks.summary(),
