@@ -174,16 +174,98 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_gemm(args):
+    """Secondary workload (not the default bench line): the paper's bf16 GEMM C = A B^T,
+    A 8192x5120, B 7168x5120, seeded synthetic N(0,1) inputs.  One step = one GEMM."""
+    M, N, K = 8192, 7168, 5120
+    flops = 2.0 * M * N * K
+    a_bits = W.gen_tensor_bits(7, W.TENSOR_Q, (M, K))
+    b_bits = W.gen_tensor_bits(7, W.TENSOR_K, (N, K))
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return
+        from oracle import gemm as G
+        a64, b64 = W.bf16_bits_to_f64(a_bits), W.bf16_bits_to_f64(b_bits)
+        rows = 256
+        secs = []
+        for i in range(args.warmup + args.steps):
+            t0 = time.perf_counter()
+            G.gemm_nt_rows(a64, b64, range(i * rows % M, i * rows % M + rows))
+            if i >= args.warmup:
+                secs.append(time.perf_counter() - t0)
+        value = 2.0 * rows * N * K * len(secs) / sum(secs) / 1e12
+        print(json.dumps({"impl": "reference", "metric": "GEMM TFLOPS (bf16 inputs)", "value": value, "unit": "TFLOP/s",
+                          "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": {"workload": "gemm 8192x7168x5120", "note": f"fp64 numpy oracle, {rows} output rows per step"},
+                          "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+                                           "sample": f"{rows} of {M} output rows per step"},
+                          "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}), flush=True)
+        return
+    from paper_2608_17379_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GEMM path has no CPU fallback")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    to_t = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    a_h, b_h = to_t(a_bits).pin_memory(), to_t(b_bits).pin_memory()
+    a, b = a_h.cuda(), b_h.cuda()
+    c = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    c_h = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    for _ in range(max(args.warmup, 3)):
+        binding.gemm_bf16_nt(a, b, c=c)
+    torch.cuda.synchronize()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    K_ = args.steps
+    with ClockSampler(0) as clocks:
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(K_):
+            binding.gemm_bf16_nt(a, b, c=c)
+        e1.record()
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / K_
+    s0, s1 = ev(), ev()
+    s0.record()
+    for _ in range(3):
+        a.copy_(a_h, non_blocking=True); b.copy_(b_h, non_blocking=True)
+        binding.gemm_bf16_nt(a, b, c=c)
+        c_h.copy_(c, non_blocking=True)
+    s1.record()
+    torch.cuda.synchronize()
+    e2e_ms = s0.elapsed_time(s1) / 3
+    assert binding.query_status() == (0, 0)
+    peaks = measured_peaks()
+    tf = flops / (ms * 1e-3) / 1e12
+    peak = float(peaks["bf16_tflops"] if K_ <= 30 else peaks["bf16_tflops_sustained"])
+    line = {"metric": "GEMM TFLOPS (bf16, device-timed)", "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": K_,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "gemm C=A*B^T 8192x7168x5120", "l2": "A+B+C = 274 MB exceed the 126 MB L2; no flush"},
+            "roofline": {"bound": "tensor", "kernel": "gemm_bf16_nt_kernel", "achieved": tf, "peak": peak,
+                         "unit": "TFLOP/s", "frac": tf / peak,
+                         "peak_source": f"{peaks['_source']} bf16 " + ("burst" if K_ <= 30 else "sustained"),
+                         "traffic": None},
+            "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": (M + N) * K * 2, "d2h_bytes_per_step": M * N * 2},
+            "gpu_launches": K_, "clocks": clocks.summary()}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c3", choices=list(W.CONFIG_NAMES))
+    ap.add_argument("--config", default="c3", choices=list(W.CONFIG_NAMES) + ["gemm"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.config == "gemm":
+        run_gemm(args)
+        return
     w = W.config(args.config)
 
     if args.impl == "reference":

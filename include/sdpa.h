@@ -154,6 +154,17 @@ int sdpa_fwd_bwd_host(const void* q, const void* k, const void* v, const void* d
 int sdpa_bwd_profile_events(void* ev_main_start, void* ev_main_stop);
 
 /*
+ * bf16 GEMM C = A B^T (paper, appendix "Workloads": the fifth primary workload, C = A B^T at BF16 with
+ * A 8192x5120, B 7168x5120, C 8192x7168).  a [M,K], b [N,K], c [M,N]: row-major contiguous bf16
+ * DEVICE pointers, 16-byte aligned, caller-owned; products are accumulated in fp32 on the tensor cores
+ * and c is rounded to bf16 (nearest even) and overwritten.  Any M >= 0; N and K must be multiples of
+ * 8 (16-byte row pitches), K > 0 unless the output is empty; other shapes return SDPA_ERR_SHAPE.
+ * Asynchronous on `stream`; nothing is allocated.  Errors and the device status word are those of
+ * the other entry points.
+ */
+int gemm_bf16_nt(const void* a, const void* b, void* c, int M, int N, int K, void* stream);
+
+/*
  * Waits for `stream`, then returns the current device's status word (0 = no device-side problem
  * since the last query; otherwise an SDPA_STATUS_* code) and clears it.  *site (may be null)
  * receives an internal identifier of the wait that gave up.  Returns SDPA_ERR_CUDA if the

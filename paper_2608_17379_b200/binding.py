@@ -18,7 +18,7 @@ _LIB = None
 SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
-           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch")
+           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt")
 
 
 class SdpaError(RuntimeError):
@@ -49,6 +49,8 @@ def load():
     lib.sdpa_bwd_profile_events.argtypes = [vp, vp]
     lib.sdpa_bwd_static_scratch.restype = ci
     lib.sdpa_bwd_static_scratch.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp]
+    lib.gemm_bf16_nt.restype = ci
+    lib.gemm_bf16_nt.argtypes = [vp, vp, vp, ci, ci, ci, vp]
     lib.sdpa_query_status.restype = ci
     lib.sdpa_query_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.sdpa_status_string.restype = ctypes.c_char_p
@@ -149,7 +151,7 @@ def sdpa_bwd_static_scratch(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, 
                                      int(max_seqlen), _stream_ptr(stream))
     if rc == SDPA_ERR_STATIC_SCRATCH:
         return rc
-    _check(rc, "sdpa_bwd_static_scratch")
+    _check(rc, "sdpa_bwd_static_scratch", "gemm_bf16_nt")
     return rc
 
 
@@ -179,6 +181,19 @@ def bwd_profile_events(start=None, stop=None):
     s = 0 if start is None else int(start.cuda_event)
     e = 0 if stop is None else int(stop.cuda_event)
     _check(load().sdpa_bwd_profile_events(s, e), "sdpa_bwd_profile_events")
+
+
+def gemm_bf16_nt(a, b, c=None, stream=None):
+    """c [M,N] = a [M,K] @ b [N,K]^T, bf16 CUDA tensors, fp32 accumulation on the tensor cores."""
+    lib = load()
+    assert a.dtype == torch.bfloat16 and b.dtype == torch.bfloat16 and a.is_contiguous() and b.is_contiguous()
+    M, K = a.shape
+    N = b.shape[0]
+    assert b.shape[1] == K
+    if c is None:
+        c = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
+    _check(lib.gemm_bf16_nt(_ptr(a), _ptr(b), _ptr(c), M, N, K, _stream_ptr(stream)), "gemm_bf16_nt")
+    return c
 
 
 def query_status(stream=None):

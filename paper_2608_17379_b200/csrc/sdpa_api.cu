@@ -8,6 +8,7 @@
 
 #include "bwd_kernel.cuh"
 #include "fwd_kernel.cuh"
+#include "gemm_kernel.cuh"
 
 namespace sdpa {
 
@@ -78,6 +79,8 @@ static int device_state(DeviceState** out) {
                                                BwdCfg<128>::kSmemBytes));
             SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                BwdCfg<64>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(gemm_bf16_nt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               GemmCfg::kSmemBytes));
         }
         st.ready = true;
     }
@@ -347,6 +350,47 @@ extern "C" int sdpa_fwd_bwd_host(const void* q, const void* k, const void* v, co
     SDPA_CUDA_TRY(cudaMemcpyAsync(dq, d_dq, q_bytes, cudaMemcpyDeviceToHost, s));
     SDPA_CUDA_TRY(cudaMemcpyAsync(dk, d_dk, k_bytes, cudaMemcpyDeviceToHost, s));
     SDPA_CUDA_TRY(cudaMemcpyAsync(dv, d_dv, k_bytes, cudaMemcpyDeviceToHost, s));
+    return SDPA_OK;
+}
+
+// Tensor map over a row-major bf16 matrix [rows, cols]: dims {cols, rows}, box {64, box_rows}, 128B swizzle.
+static int make_map_2d(CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = static_cast<int>(r);
+        return SDPA_ERR_CUDA;
+    }
+    return SDPA_OK;
+}
+
+extern "C" int gemm_bf16_nt(const void* a, const void* b, void* c, int M, int N, int K, void* stream) {
+    if (M < 0 || N < 0 || K < 0) return SDPA_ERR_SHAPE;
+    if ((K % 8) != 0 || (N % 8) != 0) return SDPA_ERR_SHAPE;  // 16-byte row pitches and 16-byte output vectors
+    if (M == 0 || N == 0) return SDPA_OK;
+    if (K == 0) return SDPA_ERR_SHAPE;
+    if (!a || !b || !c) return SDPA_ERR_NULL;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(c)) return SDPA_ERR_ALIGN;
+    DeviceState* st = nullptr;
+    int rc = device_state(&st);
+    if (rc != SDPA_OK) return rc;
+    CUtensorMap ma, mb;
+    if ((rc = make_map_2d(&ma, a, M, K, GemmCfg::BM)) != SDPA_OK) return rc;
+    if ((rc = make_map_2d(&mb, b, N, K, GemmCfg::BN)) != SDPA_OK) return rc;
+    GemmParams p;
+    p.c = static_cast<__nv_bfloat16*>(c);
+    p.status = st->status_ptr;
+    p.M = M; p.N = N; p.K = K;
+    const long long tiles = static_cast<long long>((M + GemmCfg::BM - 1) / GemmCfg::BM) * ((N + GemmCfg::BN - 1) / GemmCfg::BN);
+    if (tiles > 2147483647ll) return SDPA_ERR_SHAPE;
+    const unsigned grid = static_cast<unsigned>(tiles < st->num_sms ? tiles : st->num_sms);
+    gemm_bf16_nt_kernel<<<grid, GemmCfg::kThreads, GemmCfg::kSmemBytes, static_cast<cudaStream_t>(stream)>>>(ma, mb, p);
+    SDPA_CUDA_TRY(cudaGetLastError());
     return SDPA_OK;
 }
 
