@@ -17,6 +17,10 @@
 #pragma once
 #include "ptx.cuh"
 
+#ifndef SDPA_TR
+#define SDPA_TR(role, it, k) do { } while (0)
+#endif
+
 namespace sdpa {
 
 struct FwdParams {
@@ -142,8 +146,10 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int n = n_kv[t];
         bool ok = true;
         for (int j = 0; j < n && ok; ++j) {
+            if (row_in_tile == 0) SDPA_TR(t, j, 0);
             ok = mbar_wait_warp(&s_full[t], j & 1, ctl, kSiteSFull);
             if (!ok) break;
+            if (row_in_tile == 0) SDPA_TR(t, j, 1);
             tc_fence_after();
             float s[128];
 #pragma unroll
@@ -154,6 +160,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
             }
             tmem_wait_ld();
+            if (row_in_tile == 0) SDPA_TR(t, j, 2);
             const int key0 = j * 128;
             const bool diag = p.causal && (key0 + 127 > q_start + t * 128);
             if (diag || key0 + 128 > L) {
@@ -185,6 +192,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                 }
             }
+            if (row_in_tile == 0) SDPA_TR(t, j, 3);
             const float neg_m = -m * p.scale_log2;
             float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
@@ -201,9 +209,11 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tmem_st_x32(tS + c * 32, r);
             }
             l += sum0 + sum1;
+            if (row_in_tile == 0) SDPA_TR(t, j, 4);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&p_full[t]);
+            if (row_in_tile == 0) SDPA_TR(t, j, 5);
         }
         if (ok && n > 0) ok = mbar_wait_warp(&o_full[t], 0, ctl, kSiteOFull);
         if (ok && n > 0) {
@@ -313,8 +323,10 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
                 for (int j = 0; j < n_iter && ok; ++j) {
                     const int st_v = it % S;
+                    SDPA_TR(2, j, 0);
                     ok = mbar_wait(&kv_full[st_v], (it / S) & 1, ctl, kSiteKvFull);
                     if (!ok) break;
+                    SDPA_TR(2, j, 1);
                     ++it;
                     const bool have_next = (j + 1) < n_iter;
                     const int st_k = it % S;
@@ -323,6 +335,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         if (j >= n_kv[t]) continue;
                         ok = mbar_wait(&p_full[t], j & 1, ctl, kSitePFull);
                         if (!ok) break;
+                        SDPA_TR(2, j, 2 + 2 * t);
                         tc_fence_after();
                         issue_pv(t, st_v, j > 0);
                         if (j + 1 < n_kv[t]) {
@@ -337,6 +350,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         } else {
                             umma_commit(&o_full[t]);
                         }
+                        SDPA_TR(2, j, 3 + 2 * t);
                     }
                     if (!ok) break;
                     umma_commit(&kv_empty[st_v]);
