@@ -165,6 +165,15 @@ int sdpa_bwd_profile_events(void* ev_main_start, void* ev_main_stop);
 int gemm_bf16_nt(const void* a, const void* b, void* c, int M, int N, int K, void* stream);
 
 /*
+ * Self-test of the failure path (the paper's profiling service isolates kernels that "may crash, hang,
+ * or corrupt subsequent measurements", section "Multi-turn Evaluation Protocol"; this library instead
+ * bounds every device-side wait).  Launches one warp that waits on a barrier nobody signals, with a
+ * limit of `limit_cycles` SM cycles (1 .. 4e9).  The wait gives up, the kernel returns normally, and
+ * the next sdpa_query_status reports SDPA_STATUS_TIMEOUT with site 99; the context stays usable.
+ */
+int sdpa_selftest_wait_timeout(long long limit_cycles, void* stream);
+
+/*
  * Waits for `stream`, then returns the current device's status word (0 = no device-side problem
  * since the last query; otherwise an SDPA_STATUS_* code) and clears it.  *site (may be null)
  * receives an internal identifier of the wait that gave up.  Returns SDPA_ERR_CUDA if the

@@ -18,7 +18,7 @@ _LIB = None
 SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
-           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt")
+           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout")
 
 
 class SdpaError(RuntimeError):
@@ -49,6 +49,8 @@ def load():
     lib.sdpa_bwd_profile_events.argtypes = [vp, vp]
     lib.sdpa_bwd_static_scratch.restype = ci
     lib.sdpa_bwd_static_scratch.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp]
+    lib.sdpa_selftest_wait_timeout.restype = ci
+    lib.sdpa_selftest_wait_timeout.argtypes = [ctypes.c_longlong, vp]
     lib.gemm_bf16_nt.restype = ci
     lib.gemm_bf16_nt.argtypes = [vp, vp, vp, ci, ci, ci, vp]
     lib.sdpa_query_status.restype = ci
@@ -151,7 +153,7 @@ def sdpa_bwd_static_scratch(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, 
                                      int(max_seqlen), _stream_ptr(stream))
     if rc == SDPA_ERR_STATIC_SCRATCH:
         return rc
-    _check(rc, "sdpa_bwd_static_scratch", "gemm_bf16_nt")
+    _check(rc, "sdpa_bwd_static_scratch")
     return rc
 
 

@@ -613,7 +613,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         t_idle = clock64();
                     } else if (*ctl.abort) {
                         ok = false;
-                    } else if (clock64() - t_idle > SDPA_WAIT_LIMIT_CYCLES) {
+                    } else if (clock64() - t_idle > ctl.limit) {
                         *ctl.abort = 1;
                         atomicCAS(ctl.g_status, 0, (kBSiteDqEmpty << 8) | kStatusTimeout);
                         ok = false;

@@ -49,6 +49,11 @@ struct FwdCfg {
     static constexpr int kKSteps = D / 16;                       // k-steps of S = Q K^T
 };
 
+#ifndef SDPA_FWD_EMUL_PAIRS
+#define SDPA_FWD_EMUL_PAIRS 2
+#endif
+constexpr int kEmulPairs = SDPA_FWD_EMUL_PAIRS;  // of every 8 score pairs, how many take the polynomial exp2
+
 enum FwdSite {
     kSiteQFull = 1, kSiteKvFull = 2, kSiteKvEmpty = 3, kSiteSFull = 4, kSitePFull = 5, kSiteOFull = 6,
     kSiteDrain = 7
@@ -169,9 +174,17 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int c = 0; c < 128; ++c)
                     if (key0 + c > lim) s[c] = -INFINITY;
             }
-            float mx = s[0];
+            float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
 #pragma unroll
-            for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+            for (int c = 4; c < 124; c += 8) {
+                mx0 = max3(mx0, s[c], s[c + 1]);
+                mx1 = max3(mx1, s[c + 2], s[c + 3]);
+                mx2 = max3(mx2, s[c + 4], s[c + 5]);
+                mx3 = max3(mx3, s[c + 6], s[c + 7]);
+            }
+            mx0 = max3(mx0, s[124], s[125]);
+            mx1 = max3(mx1, s[126], s[127]);
+            const float mx = fmaxf(max3(mx0, mx1, mx2), mx3);
             if (j == 0) {
                 m = mx;
             } else {
@@ -193,22 +206,39 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
             }
             if (row_in_tile == 0) SDPA_TR(t, j, 3);
+            // p = exp2(s * c - m * c) on pairs of scores: one packed FMA, then either two SFU ex2 or (for
+            // kEmulPairs of every eight pairs) the FMA-pipe polynomial, so the SFU is not the only exp unit.
             const float neg_m = -m * p.scale_log2;
-            float sum0 = 0.f, sum1 = 0.f;
+            const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2), nm2 = pack_f32x2(neg_m, neg_m);
+            uint64_t sum_a = pack_f32x2(0.f, 0.f), sum_b = pack_f32x2(0.f, 0.f);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t r[32];
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    const float e0 = fast_exp2(fmaf(s[c * 64 + 2 * i], p.scale_log2, neg_m));
-                    const float e1 = fast_exp2(fmaf(s[c * 64 + 2 * i + 1], p.scale_log2, neg_m));
-                    sum0 += e0;
-                    sum1 += e1;
+                    const uint64_t x2 = fma_f32x2(pack_f32x2(s[c * 64 + 2 * i], s[c * 64 + 2 * i + 1]), c2, nm2);
+                    uint64_t e2;
+                    if ((i & 7) < kEmulPairs) {
+                        e2 = exp2_poly_x2(x2);
+                    } else {
+                        float x0, x1;
+                        unpack_f32x2(x2, x0, x1);
+                        e2 = pack_f32x2(fast_exp2(x0), fast_exp2(x1));
+                    }
+                    if (i & 1) sum_b = add_f32x2(sum_b, e2);
+                    else sum_a = add_f32x2(sum_a, e2);
+                    float e0, e1;
+                    unpack_f32x2(e2, e0, e1);
                     r[i] = pack_bf16x2(e0, e1);
                 }
                 tmem_st_x32(tS + c * 32, r);
             }
-            l += sum0 + sum1;
+            {
+                float a0, a1, b0, b1;
+                unpack_f32x2(sum_a, a0, a1);
+                unpack_f32x2(sum_b, b0, b1);
+                l += (a0 + a1) + (b0 + b1);
+            }
             if (row_in_tile == 0) SDPA_TR(t, j, 4);
             tmem_wait_st();
             tc_fence_before();

@@ -70,6 +70,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 struct WaitCtl {
     int* g_status;        // global status word (0 = ok); first failure wins
     volatile int* abort;  // shared-memory flag; once set every wait returns false at once
+    long long limit = SDPA_WAIT_LIMIT_CYCLES;  // cycles after which a wait gives up
 };
 
 // Bounded wait.  Returns false if the wait was abandoned (timeout here or abort elsewhere).
@@ -80,7 +81,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0u) {
             if (*ctl.abort) return false;
-            if (clock64() - t0 > SDPA_WAIT_LIMIT_CYCLES) {
+            if (clock64() - t0 > ctl.limit) {
                 *ctl.abort = 1;
                 atomicCAS(ctl.g_status, 0, (site << 8) | kStatusTimeout);
                 return false;
@@ -277,6 +278,52 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+
+// ------------------------------------------------------------------ packed fp32 pairs, 3-input max
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// 2^x for a pair of values on the FMA pipe instead of the SFU: round(x) through the 1.5*2^23 trick,
+// a cubic for 2^f on f in [-0.5, 0.5] (max relative error 7.5e-5, far below the bf16 rounding of P),
+// and the exponent added as an integer.  Inputs are clamped to >= -125 (result ~2e-38 instead of 0).
+__device__ __forceinline__ uint64_t exp2_poly_x2(uint64_t x2) {
+    float x0, x1;
+    unpack_f32x2(x2, x0, x1);
+    x2 = pack_f32x2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t t2 = add_f32x2(x2, pack_f32x2(12582912.f, 12582912.f));       // low mantissa bits = round(x)
+    const uint64_t r2 = add_f32x2(t2, pack_f32x2(-12582912.f, -12582912.f));     // round(x) as a float
+    const uint64_t f2 = fma_f32x2(r2, pack_f32x2(-1.f, -1.f), x2);                // x - round(x)
+    uint64_t p2 = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), f2, pack_f32x2(0.2426111251f, 0.2426111251f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.6932609677f, 0.6932609677f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.9999280572f, 0.9999280572f));
+    float t0, t1, p0, p1;
+    unpack_f32x2(t2, t0, t1);
+    unpack_f32x2(p2, p0, p1);
+    // (bits of 1.5*2^23) << 23 is 0 modulo 2^32, so shifting the whole word adds round(x) to the exponent
+    const uint32_t e0 = __float_as_uint(p0) + (__float_as_uint(t0) << 23);
+    const uint32_t e1 = __float_as_uint(p1) + (__float_as_uint(t1) << 23);
+    return pack_f32x2(__uint_as_float(e0), __uint_as_float(e1));
 }
 
 // Byte offset of element (row, col16) inside a 128B-swizzled tile whose rows are 128 bytes:

@@ -394,6 +394,32 @@ extern "C" int gemm_bf16_nt(const void* a, const void* b, void* c, int M, int N,
     return SDPA_OK;
 }
 
+// One warp waits on an mbarrier that nobody ever arrives at: exercises the bounded wait, the status
+// word and the clean exit of a CTA without faulting or hanging the GPU.
+__global__ void sdpa_selftest_wait_kernel(int* status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    WaitCtl ctl{status, &abort_flag, limit_cycles};
+    const bool ok = mbar_wait_warp(&bar, 0, ctl, 99);
+    (void)ok;
+}
+
+extern "C" int sdpa_selftest_wait_timeout(long long limit_cycles, void* stream) {
+    if (limit_cycles < 1 || limit_cycles > 4000000000ll) return SDPA_ERR_SHAPE;  // at most ~2 s
+    DeviceState* st = nullptr;
+    int rc = device_state(&st);
+    if (rc != SDPA_OK) return rc;
+    sdpa_selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(st->status_ptr, limit_cycles);
+    SDPA_CUDA_TRY(cudaGetLastError());
+    return SDPA_OK;
+}
+
 extern "C" int sdpa_query_status(void* stream, int* site) {
     DeviceState* st = nullptr;
     int rc = device_state(&st);

@@ -231,6 +231,17 @@ def test_bad_cu_seqlens_is_reported_not_faulted():
     assert binding.query_status() == (0, 0)  # cleared by the query
 
 
+def test_a_wait_that_runs_out_reports_timeout_and_the_context_survives():
+    """Failure detection without a GPU fault: a barrier nobody signals, a one-millisecond limit."""
+    lib = binding.load()
+    assert binding.query_status() == (0, 0)
+    assert lib.sdpa_selftest_wait_timeout(2_000_000, None) == 0
+    st, site = binding.query_status()
+    assert (st, site) == (1, 99)
+    assert binding.query_status() == (0, 0)
+    run_and_compare(TL.random_workload((200,), 2, 2, 64, True, seed=61))  # the library still works
+
+
 def test_host_buffer_entry_point_matches_device_entry_points():
     w = TL.random_workload((333, 200), 4, 2, 128, True, seed=60)
     qb, kb, vb, dob = W.make_inputs(w)
