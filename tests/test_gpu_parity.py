@@ -76,7 +76,7 @@ def test_paper_ragged_shape():
 
 
 # ------------------------------------------------------------------ full-size configurations, sampled slices
-@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c4c", "c5"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c4c", "c5", "mha", "mha_causal", "mha_d64"])
 def test_full_configs_on_sampled_slices(name):
     """The five benchmark configurations in the launch configuration the bench times; the oracle
     checks complete O/LSE/dQ/dK/dV of independent (sequence, kv-head) slices."""
@@ -86,6 +86,8 @@ def test_full_configs_on_sampled_slices(name):
         slices = [(int(np.argmin(lens)), 0), (int(np.argsort(lens)[len(lens) // 2]), w.Hkv - 1)]
     elif name in ("c4", "c4c"):
         slices = [(0, 5)]
+    elif name.startswith("mha"):
+        slices = [(1, 17)]
     else:
         slices = [(0, 0), (w.B - 1, w.Hkv - 1)]
     run_and_compare(w, slices)
