@@ -72,6 +72,26 @@ int sdpa_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
              int total_tokens, int max_seqlen, void* stream);
 
 /*
+ * Forward pass over a paged KV cache (paper, appendix "Generalization attention workloads": GQA paged
+ * causal prefill and paged decode, page size 1, key/value rows addressed through a list of page
+ * indices; each returns a bf16 attention output and an fp32 log-sum-exp).
+ *   q            : bf16 [total_q, Hq, D], packed by cu_seqlens_q (int32 [B+1], device)
+ *   k_cache, v_cache : bf16 [num_pages, Hkv, D], one token per page
+ *   kv_indptr    : int32 [B+1] (device); sequence b owns kv_indices[kv_indptr[b] .. kv_indptr[b+1]-1]
+ *   kv_indices   : int32 page numbers in [0, num_pages), in key order
+ *   o, lse       : as sdpa_fwd ([total_q, Hq, D] bf16, [Hq, total_q] fp32)
+ * A sequence may have more keys than queries (Lk >= Lq, e.g. decode: Lq = 1).  With causal != 0 the
+ * mask is aligned to the end: query i sees keys 0 .. i + (Lk - Lq); with causal == 0 all Lk keys.
+ * A sequence with fewer keys than queries, or a page index outside [0, num_pages), is reported as
+ * SDPA_STATUS_BAD_CU_SEQLENS (no out-of-range read happens).  Other conventions, supported D, return
+ * codes: as sdpa_fwd.
+ */
+int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                   const int32_t* cu_seqlens_q, const int32_t* kv_indptr, const int32_t* kv_indices,
+                   int B, int Hq, int Hkv, int D, int causal, float scale, int total_q,
+                   int max_seqlen_q, int num_pages, void* stream);
+
+/*
  * Bytes of scratch sdpa_bwd needs for these sizes (fp32 dQ accumulator [T,Hq,D] plus the fp32
  * row terms D_i [Hq,T]); 0 on invalid arguments.  The workspace must be 256-byte aligned device
  * memory; its contents on entry do not matter and are unspecified on exit.

@@ -18,7 +18,7 @@ _LIB = None
 SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
-           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout")
+           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout", "sdpa_fwd_paged")
 
 
 class SdpaError(RuntimeError):
@@ -51,6 +51,8 @@ def load():
     lib.sdpa_bwd_static_scratch.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp]
     lib.sdpa_selftest_wait_timeout.restype = ci
     lib.sdpa_selftest_wait_timeout.argtypes = [ctypes.c_longlong, vp]
+    lib.sdpa_fwd_paged.restype = ci
+    lib.sdpa_fwd_paged.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, cf, ci, ci, ci, vp]
     lib.gemm_bf16_nt.restype = ci
     lib.gemm_bf16_nt.argtypes = [vp, vp, vp, ci, ci, ci, vp]
     lib.sdpa_query_status.restype = ci
@@ -183,6 +185,26 @@ def bwd_profile_events(start=None, stop=None):
     s = 0 if start is None else int(start.cuda_event)
     e = 0 if stop is None else int(stop.cuda_event)
     _check(load().sdpa_bwd_profile_events(s, e), "sdpa_bwd_profile_events")
+
+
+def sdpa_fwd_paged(q, k_cache, v_cache, cu_seqlens_q, kv_indptr, kv_indices, max_seqlen_q: int, causal: bool,
+                   scale: float, o=None, lse=None, stream=None):
+    """Forward over a page-size-1 KV cache: q [Tq,Hq,D], k_cache/v_cache [num_pages,Hkv,D] bf16 CUDA
+    tensors; cu_seqlens_q, kv_indptr int32 [B+1] and kv_indices int32 on the device."""
+    lib = load()
+    T, Hq, Hkv, D = _dims(q, k_cache)
+    B = cu_seqlens_q.numel() - 1
+    for t in (cu_seqlens_q, kv_indptr, kv_indices):
+        assert t.dtype == torch.int32 and t.is_cuda
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((Hq, T), dtype=torch.float32, device=q.device)
+    rc = lib.sdpa_fwd_paged(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(cu_seqlens_q),
+                            _ptr(kv_indptr), _ptr(kv_indices), B, Hq, Hkv, D, int(bool(causal)), float(scale), T,
+                            int(max_seqlen_q), int(k_cache.shape[0]), _stream_ptr(stream))
+    _check(rc, "sdpa_fwd_paged")
+    return o, lse
 
 
 def gemm_bf16_nt(a, b, c=None, stream=None):

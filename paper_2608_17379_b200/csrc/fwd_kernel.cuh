@@ -24,7 +24,13 @@
 namespace sdpa {
 
 struct FwdParams {
-    const int32_t* cu_seqlens;
+    const int32_t* cu_seqlens;   // query rows of sequence b: cu_seqlens[b] .. cu_seqlens[b+1]-1
+    // paged variant only: keys/values of sequence b are the cache rows kv_indices[kv_indptr[b] + j]
+    const int32_t* kv_indptr;
+    const int32_t* kv_indices;
+    const __nv_bfloat16* k_cache;  // [num_pages, Hkv, D], page size 1
+    const __nv_bfloat16* v_cache;
+    int num_pages;
     __nv_bfloat16* o;
     float* lse;
     int* status;
@@ -59,7 +65,21 @@ enum FwdSite {
     kSiteDrain = 7
 };
 
-template <int D>
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead of reading.
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// kPaged = false: K/V are packed [T, Hkv, D] tensors loaded by TMA, keys and queries of a sequence have
+// equal length.  kPaged = true: K/V rows are gathered from a page-size-1 cache through a page table,
+// a sequence may have more keys than queries, and a causal query i sees keys 0 .. i + (Lk - Lq).
+template <int D, bool kPaged>
 __global__ void __launch_bounds__(384, 1)
 sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
@@ -79,13 +99,23 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     const int q_start = pair * 256;
     if (q_start >= L) return;
+    int Lk = L, kbase = 0;  // number of keys of this sequence; first entry of its page list
+    if (kPaged) {
+        kbase = p.kv_indptr[b];
+        Lk = p.kv_indptr[b + 1] - kbase;
+        if (Lk < L || kbase < 0) {  // fewer keys than queries would leave fully masked rows
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
+            return;
+        }
+    }
+    const int off = Lk - L;  // causal alignment: the last query sees the last key
 
     int n_kv[2];
-    const int n_kv_all = (L + 127) >> 7;
+    const int n_kv_all = (Lk + 127) >> 7;
     {
         const bool has1 = (q_start + 128) < L;
-        n_kv[0] = p.causal ? (q_start >> 7) + 1 : n_kv_all;
-        n_kv[1] = has1 ? (p.causal ? ((q_start + 128) >> 7) + 1 : n_kv_all) : 0;
+        n_kv[0] = p.causal ? min(n_kv_all, ((q_start + 127 + off) >> 7) + 1) : n_kv_all;
+        n_kv[1] = has1 ? (p.causal ? min(n_kv_all, ((q_start + 255 + off) >> 7) + 1) : n_kv_all) : 0;
     }
     const int n_iter = max(n_kv[0], n_kv[1]);
 
@@ -117,7 +147,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             mbar_init(&o_full[i], 1);
         }
         for (int i = 0; i < S; ++i) {
-            mbar_init(&kv_full[i], 1);
+            mbar_init(&kv_full[i], kPaged ? 32 : 1);  // TMA transaction, or the 32 gathering lanes
             mbar_init(&kv_empty[i], 1);
         }
         mbar_init(drain, 1);
@@ -167,9 +197,9 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tmem_wait_ld();
             if (row_in_tile == 0) SDPA_TR(t, j, 2);
             const int key0 = j * 128;
-            const bool diag = p.causal && (key0 + 127 > q_start + t * 128);
-            if (diag || key0 + 128 > L) {
-                const int lim = p.causal ? min(row, L - 1) : (L - 1);  // last allowed key
+            const bool diag = p.causal && (key0 + 127 > q_start + t * 128 + off);
+            if (diag || key0 + 128 > Lk) {
+                const int lim = p.causal ? min(row + off, Lk - 1) : (Lk - 1);  // last allowed key
 #pragma unroll
                 for (int c = 0; c < 128; ++c)
                     if (key0 + c > lim) s[c] = -INFINITY;
@@ -271,7 +301,73 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else {
         setmaxnreg_dec<80>();
-        if (warp == 9) {
+        if (warp == 9 && kPaged) {
+            // -------------------------------------------------------- gathering producer (all 32 lanes)
+            // Lane l copies key rows l, l+32, l+64, l+96 of each tile from the page-size-1 cache with
+            // 16-byte cp.async into the same 128B-swizzled layout a TMA load would produce; rows past
+            // the sequence end are zero-filled (a masked P of exactly 0 must not meet garbage in V).
+            const int lane = tid & 31;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(&q_full[0], Cfg::kTileBytes);
+#pragma unroll
+                for (int a = 0; a < D / 64; ++a) tma_load_3d(sQ + a * Cfg::kAtomBytes, &map_q, &q_full[0], a * 64, h, r0 + q_start);
+                if (n_kv[1] > 0) {
+                    mbar_arrive_expect_tx(&q_full[1], Cfg::kTileBytes);
+#pragma unroll
+                    for (int a = 0; a < D / 64; ++a)
+                        tma_load_3d(sQ + Cfg::kTileBytes + a * Cfg::kAtomBytes, &map_q, &q_full[1], a * 64, h,
+                                    r0 + q_start + 128);
+                }
+            }
+            bool ok = true;
+            int it = 0;
+            int pending = -1;  // ring slot whose copies are in flight (one group deep)
+            for (int j = 0; j < n_iter && ok; ++j) {
+                int page[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int key = j * 128 + lane + 32 * i;
+                    int pg = -1;
+                    if (key < Lk) {
+                        pg = p.kv_indices[kbase + key];
+                        if (pg < 0 || pg >= p.num_pages) {  // never read outside the cache
+                            atomicCAS(p.status, 0, kStatusBadCuSeqlens);
+                            pg = -1;
+                        }
+                    }
+                    page[i] = pg;
+                }
+                for (int kv = 0; kv < 2 && ok; ++kv, ++it) {
+                    const int st = it % S;
+                    ok = mbar_wait_warp(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
+                    if (!ok) break;
+                    uint8_t* dst = sRing + st * Cfg::kTileBytes;
+                    const __nv_bfloat16* cache = kv == 0 ? p.k_cache : p.v_cache;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = lane + 32 * i;
+                        const bool have = page[i] >= 0;
+                        const __nv_bfloat16* src = cache + (static_cast<size_t>(have ? page[i] : 0) * p.Hkv + g) * D;
+#pragma unroll
+                        for (int c = 0; c < D / 8; ++c)
+                            cp_async_16(dst + (c >> 3) * Cfg::kAtomBytes + sw128_offset(row, c & 7), src + c * 8,
+                                        have ? 16u : 0u);
+                    }
+                    cp_async_commit();
+                    if (pending >= 0) {
+                        cp_async_wait<1>();          // the previous slot's copies have landed
+                        fence_proxy_async_smem();    // make them visible to the tensor core's reads
+                        mbar_arrive(&kv_full[pending]);
+                    }
+                    pending = st;
+                }
+            }
+            cp_async_wait<0>();
+            if (ok && pending >= 0) {
+                fence_proxy_async_smem();
+                mbar_arrive(&kv_full[pending]);
+            }
+        } else if (warp == 9) {
             // -------------------------------------------------------- TMA producer
             if (elect_one()) {
                 int it = 0;

@@ -71,9 +71,13 @@ static int device_state(DeviceState** out) {
             SDPA_CUDA_TRY(cudaGetSymbolAddress(&sym, g_status_word));
             st.status_ptr = static_cast<int*>(sym);
             SDPA_CUDA_TRY(cudaMemset(st.status_ptr, 0, sizeof(int)));
-            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                FwdCfg<128>::kSmemBytes));
-            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               FwdCfg<64>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               FwdCfg<128>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                FwdCfg<64>::kSmemBytes));
             SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                BwdCfg<128>::kSmemBytes));
@@ -145,6 +149,7 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
 
     FwdParams p;
     p.cu_seqlens = cu_seqlens;
+    p.kv_indptr = nullptr; p.kv_indices = nullptr; p.k_cache = nullptr; p.v_cache = nullptr; p.num_pages = 0;
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
     p.status = st->status_ptr;
@@ -158,9 +163,55 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
     dim3 grid(static_cast<unsigned>(B * Hq), static_cast<unsigned>(n_pairs), 1);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (D == 128)
-        sdpa_fwd_kernel<128><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, p);
+        sdpa_fwd_kernel<128, false><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, p);
     else
-        sdpa_fwd_kernel<64><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mk, mv, p);
+        sdpa_fwd_kernel<64, false><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mk, mv, p);
+    SDPA_CUDA_TRY(cudaGetLastError());
+    return SDPA_OK;
+}
+
+extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                              const int32_t* cu_seqlens_q, const int32_t* kv_indptr, const int32_t* kv_indices, int B,
+                              int Hq, int Hkv, int D, int causal, float scale, int total_q, int max_seqlen_q,
+                              int num_pages, void* stream) {
+    int rc = check_common(cu_seqlens_q, B, Hq, Hkv, D, scale, total_q, max_seqlen_q);
+    if (rc != SDPA_OK) return rc;
+    if (num_pages < 0) return SDPA_ERR_SHAPE;
+    if (total_q == 0 || max_seqlen_q == 0) return SDPA_OK;
+    if (!q || !k_cache || !v_cache || !o || !lse || !kv_indptr || !kv_indices) return SDPA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) ||
+        (reinterpret_cast<uintptr_t>(lse) & 3u))
+        return SDPA_ERR_ALIGN;
+    if (num_pages == 0) return SDPA_ERR_SHAPE;
+    DeviceState* st = nullptr;
+    rc = device_state(&st);
+    if (rc != SDPA_OK) return rc;
+    CUtensorMap mq;
+    if ((rc = make_map(&mq, q, total_q, Hq, D, 128)) != SDPA_OK) return rc;
+    FwdParams p;
+    p.cu_seqlens = cu_seqlens_q;
+    p.kv_indptr = kv_indptr;
+    p.kv_indices = kv_indices;
+    p.k_cache = static_cast<const __nv_bfloat16*>(k_cache);
+    p.v_cache = static_cast<const __nv_bfloat16*>(v_cache);
+    p.num_pages = num_pages;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
+    p.status = st->status_ptr;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.T = total_q;
+    p.causal = causal ? 1 : 0;
+    p.max_seqlen = max_seqlen_q;
+    p.scale = scale;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    const int n_pairs = (max_seqlen_q + 255) / 256;
+    if (n_pairs > 65535) return SDPA_ERR_SHAPE;
+    dim3 grid(static_cast<unsigned>(B * Hq), static_cast<unsigned>(n_pairs), 1);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the K/V tensor maps are unused by the gathering producer; the Q map stands in for them
+    if (D == 128)
+        sdpa_fwd_kernel<128, true><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mq, mq, p);
+    else
+        sdpa_fwd_kernel<64, true><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mq, mq, p);
     SDPA_CUDA_TRY(cudaGetLastError());
     return SDPA_OK;
 }
