@@ -264,3 +264,20 @@ def test_host_buffer_entry_point_matches_device_entry_points():
     assert torch.equal(dk.view(torch.int16), ref["dk"].cpu().view(torch.int16))
     assert torch.equal(dv.view(torch.int16), ref["dv"].cpu().view(torch.int16))
     assert (dq.float() - ref["dq"].cpu().float()).abs().max() <= 2e-2 * ref["dq"].float().abs().max().item()
+
+
+# ------------------------------------------------------------------ randomised shapes
+def test_random_shapes_against_the_oracle():
+    """Thirty random small problems (ragged lengths incl. zeros, MHA/GQA, both head dims, both masks)."""
+    rng = np.random.default_rng(2024)
+    for case in range(30):
+        B = int(rng.integers(1, 5))
+        lengths = [int(x) for x in rng.choice([0, 1, 63, 64, 65, 127, 128, 129, 200, 255, 256, 257, 300, 511, 700], B)]
+        if sum(lengths) == 0:
+            lengths[0] = 17
+        Hkv = int(rng.choice([1, 2, 3]))
+        G = int(rng.choice([1, 2, 4]))
+        D = int(rng.choice([64, 128]))
+        causal = bool(rng.integers(0, 2))
+        w = TL.random_workload(lengths, Hkv * G, Hkv, D, causal, seed=5000 + case, qk_mul=float(rng.choice([1.0, 2.0])))
+        run_and_compare(w)
