@@ -131,7 +131,8 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint64_t* p_full = s_full + 2;         // [2]
     uint64_t* o_full = p_full + 2;         // [2]
     uint64_t* drain = o_full + 2;          // [1]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    uint64_t* p_half = drain + 1;          // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(p_half + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x;
@@ -144,6 +145,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             mbar_init(&q_full[i], 1);
             mbar_init(&s_full[i], 1);
             mbar_init(&p_full[i], 128);
+            mbar_init(&p_half[i], 128);
             mbar_init(&o_full[i], 1);
         }
         for (int i = 0; i < S; ++i) {
@@ -262,6 +264,12 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     r[i] = pack_bf16x2(e0, e1);
                 }
                 tmem_st_x32(tS + c * 32, r);
+                if (c == 0) {
+                    // the first 64 keys of P are complete: P V may start on them while the rest is computed
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(&p_half[t]);
+                }
             }
             {
                 float a0, a1, b0, b1;
@@ -383,6 +391,9 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const int st = it % S;
                         ok = mbar_wait(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
                         if (!ok) break;
+#ifdef SDPA_EXP_NO_KV_RELOAD
+                        if (it >= S) mbar_arrive(&kv_full[st]); else
+#endif
                         load_tile(kv == 0 ? &map_k : &map_v, sRing + st * Cfg::kTileBytes, &kv_full[st], g,
                                   r0 + j * 128);
                         if (j == 0 && kv == 0 && n_kv[1] > 0)
@@ -419,14 +430,16 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         umma_ss(d, a0 + off, b0 + off, idesc_qk, kk > 0);
                     }
                 };
-                auto issue_pv = [&](int t, int st, bool accumulate) {
+                auto issue_pv = [&](int t, int st, bool accumulate, int half) {
                     const uint64_t b0 = v_desc + static_cast<uint64_t>(st * (Cfg::kTileBytes >> 4));
                     const uint32_t d = tmem + 256 + t * 128;
                     const uint32_t a = tmem + t * 128;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
+                    for (int k4 = 0; k4 < 4; ++k4) {
+                        const int kk = half * 4 + k4;
                         umma_ts(d, a + kk * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_pv,
                                 (accumulate || kk > 0) ? 1u : 0u);
+                    }
                 };
                 bool ok = true;
                 int it = 0;  // ring consumer counter: K_j is item 2j, V_j is item 2j+1
@@ -459,11 +472,15 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     bool next_ready = false;
                     for (int t = 0; t < 2 && ok; ++t) {
                         if (j >= n_kv[t]) continue;
-                        ok = mbar_wait(&p_full[t], j & 1, ctl, kSitePFull);
+                        ok = mbar_wait(&p_half[t], j & 1, ctl, kSitePFull);
                         if (!ok) break;
                         SDPA_TR(2, j, 2 + 2 * t);
                         tc_fence_after();
-                        issue_pv(t, st_v, j > 0);
+                        issue_pv(t, st_v, j > 0, 0);
+                        ok = mbar_wait(&p_full[t], j & 1, ctl, kSitePFull);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(t, st_v, j > 0, 1);
                         if (j + 1 < n_kv[t]) {
                             if (!next_ready) {
                                 ok = mbar_wait(&kv_full[st_k], (it / S) & 1, ctl, kSiteKvFull);
