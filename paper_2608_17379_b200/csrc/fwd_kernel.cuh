@@ -287,21 +287,41 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (ok && n > 0) {
             tc_fence_after();
             const float inv_l = 1.0f / l;
-            __nv_bfloat16* orow = p.o + (static_cast<size_t>(r0 + row) * p.Hq + h) * D;
+            // O leaves through this tile's Q buffer (dead after the last S = Q K^T): every thread writes its
+            // normalised bf16 row there (16-byte chunks XOR-swizzled by row so the writes spread over the
+            // banks), then each warp copies its own 32 rows out with full-line stores.  Storing the rows
+            // straight from the TMEM layout (thread = row) would touch 32 different lines per store.
+            constexpr int kChunks = D / 8;             // 16-byte chunks per row
+            constexpr int kRowsPerPass = 32 / kChunks;  // rows one warp store covers
+            uint8_t* stage = sQ + t * Cfg::kTileBytes;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld_x32(tO + c * 32, r);
                 tmem_wait_ld();
-                if (valid) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(r[8 * i + 0]) * inv_l, __uint_as_float(r[8 * i + 1]) * inv_l);
-                        w.y = pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv_l, __uint_as_float(r[8 * i + 3]) * inv_l);
-                        w.z = pack_bf16x2(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
-                        w.w = pack_bf16x2(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
+                for (int i = 0; i < 4; ++i) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(r[8 * i + 0]) * inv_l, __uint_as_float(r[8 * i + 1]) * inv_l);
+                    w.y = pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv_l, __uint_as_float(r[8 * i + 3]) * inv_l);
+                    w.z = pack_bf16x2(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
+                    w.w = pack_bf16x2(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
+                    const int k = c * 4 + i;
+                    *reinterpret_cast<uint4*>(stage + row_in_tile * (D * 2) + ((k ^ (row_in_tile & 7)) << 4)) = w;
+                }
+            }
+            __syncwarp();
+            {
+                const int lane = tid & 31;
+                const int k = lane % kChunks;
+                const int rows_left = L - (q_start + t * 128);  // rows of this tile inside the sequence
+#pragma unroll
+                for (int pass = 0; pass < 32 / kRowsPerPass; ++pass) {
+                    const int rr = (warp & 3) * 32 + pass * kRowsPerPass + lane / kChunks;  // row inside the tile
+                    if (rr < rows_left) {
+                        const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * (D * 2) + ((k ^ (rr & 7)) << 4));
+                        __nv_bfloat16* dst = p.o + (static_cast<size_t>(r0 + q_start + t * 128 + rr) * p.Hq + h) * D;
+                        *reinterpret_cast<uint4*>(dst + k * 8) = w;
                     }
                 }
             }
