@@ -30,12 +30,17 @@ namespace sdpa {
 __device__ long long g_trace[5 * 32 * 8];
 #define SDPA_TR(role, it, k)                                                                   \
     do {                                                                                       \
-        if (blockIdx.x == 0 && blockIdx.y == 4 && (it) >= 8 && (it) < 40)                       \
+        if (blockIdx.y == 0 && blockIdx.x == 4 * SDPA_BWD_GROUP_CHUNK && (it) >= 8 && (it) < 40)                       \
             g_trace[((role) * 32 + ((it) - 8)) * 8 + (k)] = clock64();                         \
     } while (0)
 #else
 #define SDPA_TR(role, it, k) do { } while (0)
 #endif
+
+#ifndef SDPA_BWD_GROUP_CHUNK
+#define SDPA_BWD_GROUP_CHUNK 8
+#endif
+constexpr int kBwdGroupChunk = SDPA_BWD_GROUP_CHUNK;  // (sequence, kv head) groups whose CTAs are launched interleaved
 
 struct BwdParams {
     const int32_t* cu_seqlens;
@@ -140,7 +145,14 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const BwdParams p) {
     using Cfg = BwdCfg<D>;
     constexpr int NS = Cfg::kQStages;
-    const int bg = blockIdx.x;
+    // Launch order: the (sequence, kv head) groups are taken in chunks of kBwdGroupChunk; inside a chunk the
+    // CTAs go key tile by key tile (under a causal mask the low key tiles see the most queries, so the heavy
+    // CTAs start first), chunk after chunk.  CTAs that run at the same time therefore belong to few groups
+    // and sweep the same query heads at about the same time, which keeps the part of the fp32 dQ accumulator
+    // being reduced into inside the L2; one chunk for everything would spread a wave over all groups and
+    // every accumulator line would travel to DRAM and back once per wave.
+    const int bg = static_cast<int>(blockIdx.y) * kBwdGroupChunk + static_cast<int>(blockIdx.x) % kBwdGroupChunk;
+    if (bg >= p.B * p.Hkv) return;
     const int b = bg / p.Hkv, g = bg % p.Hkv;
     const int G = p.Hq / p.Hkv;
     const int r0 = p.cu_seqlens[b];
@@ -151,7 +163,9 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         return;
     }
     // causal: low key tiles see the most query tiles -> launch them first
-    const int jt = p.causal ? static_cast<int>(blockIdx.y) : static_cast<int>(gridDim.y) - 1 - static_cast<int>(blockIdx.y);
+    const int n_tiles_grid = static_cast<int>(gridDim.x) / kBwdGroupChunk;
+    const int jt_raw = static_cast<int>(blockIdx.x) / kBwdGroupChunk;
+    const int jt = p.causal ? jt_raw : n_tiles_grid - 1 - jt_raw;
     const int kv0 = jt * 128;
     if (kv0 >= L) return;
     const int n_qs = (L + 63) >> 6;            // 64-row query steps in the sequence
@@ -337,21 +351,43 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // group 0 writes dV, group 1 writes dK (scaled)
             const uint32_t tAcc = tmem + lane_base + (wg == 0 ? kColDV : kColDK);
             const float mul = wg == 0 ? 1.0f : p.scale;
-            __nv_bfloat16* dst = (wg == 0 ? p.dv : p.dk) + (static_cast<size_t>(r0 + key) * p.Hkv + g) * D;
+            __nv_bfloat16* out = wg == 0 ? p.dv : p.dk;
+            // The rows leave through shared memory that no MMA reads any more once dkv_full has completed: the
+            // V tile (group 0; its last reader dP^T finished before the last dS) and the first Q/dO stage
+            // (group 1; the K tile may still feed the last dQ^T).  Each thread writes its bf16 row there
+            // (16-byte chunks XOR-swizzled by row), then each warp copies its own 32 rows out with full-line
+            // stores instead of 32 different lines per store.
+            constexpr int kChunks = D / 8;
+            constexpr int kRowsPerPass = 32 / kChunks;
+            uint8_t* out_stage = wg == 0 ? sV : sQdO;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t a[32];
                 tmem_ld_x32(tAcc + c * 32, a);
                 tmem_wait_ld();
-                if (key_ok) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(a[8 * i + 0]) * mul, __uint_as_float(a[8 * i + 1]) * mul);
-                        w.y = pack_bf16x2(__uint_as_float(a[8 * i + 2]) * mul, __uint_as_float(a[8 * i + 3]) * mul);
-                        w.z = pack_bf16x2(__uint_as_float(a[8 * i + 4]) * mul, __uint_as_float(a[8 * i + 5]) * mul);
-                        w.w = pack_bf16x2(__uint_as_float(a[8 * i + 6]) * mul, __uint_as_float(a[8 * i + 7]) * mul);
-                        *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = w;
+                for (int i = 0; i < 4; ++i) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(a[8 * i + 0]) * mul, __uint_as_float(a[8 * i + 1]) * mul);
+                    w.y = pack_bf16x2(__uint_as_float(a[8 * i + 2]) * mul, __uint_as_float(a[8 * i + 3]) * mul);
+                    w.z = pack_bf16x2(__uint_as_float(a[8 * i + 4]) * mul, __uint_as_float(a[8 * i + 5]) * mul);
+                    w.w = pack_bf16x2(__uint_as_float(a[8 * i + 6]) * mul, __uint_as_float(a[8 * i + 7]) * mul);
+                    const int k = c * 4 + i;
+                    *reinterpret_cast<uint4*>(out_stage + r * (D * 2) + ((k ^ (r & 7)) << 4)) = w;
+                }
+            }
+            __syncwarp();
+            {
+                const int lane = tid & 31;
+                const int k = lane % kChunks;
+                const int rows_left = L - kv0;  // keys of this tile inside the sequence
+#pragma unroll
+                for (int pass = 0; pass < 32 / kRowsPerPass; ++pass) {
+                    const int rr = (warp & 3) * 32 + pass * kRowsPerPass + lane / kChunks;
+                    if (rr < rows_left) {
+                        const uint4 w = *reinterpret_cast<const uint4*>(out_stage + rr * (D * 2) + ((k ^ (rr & 7)) << 4));
+                        __nv_bfloat16* dst = out + (static_cast<size_t>(r0 + kv0 + rr) * p.Hkv + g) * D;
+                        *reinterpret_cast<uint4*>(dst + k * 8) = w;
                     }
                 }
             }

@@ -282,7 +282,10 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
     p.scale_log2 = scale * 1.4426950408889634f;
     const int n_kv_tiles = (max_seqlen + 127) / 128;
     if (n_kv_tiles > 65535) return SDPA_ERR_SHAPE;
-    dim3 grid(static_cast<unsigned>(B * Hkv), static_cast<unsigned>(n_kv_tiles), 1);
+    // x walks a chunk of kGroupChunk (sequence, kv head) groups key tile by key tile, y walks the chunks
+    const int n_groups = B * Hkv;
+    dim3 grid(static_cast<unsigned>(n_kv_tiles * sdpa::kBwdGroupChunk),
+              static_cast<unsigned>((n_groups + sdpa::kBwdGroupChunk - 1) / sdpa::kBwdGroupChunk), 1);
     if (tl_ev_main_start) SDPA_CUDA_TRY(cudaEventRecord(tl_ev_main_start, s));
     if (D == 128)
         sdpa_bwd_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
