@@ -37,6 +37,7 @@ struct FwdParams {
     int B, Hq, Hkv, T;
     int causal;
     int max_seqlen;
+    int head_chunk;    // (sequence, query head) pairs whose CTAs are launched interleaved
     float scale;       // softmax scale
     float scale_log2;  // scale * log2(e)
 };
@@ -86,10 +87,16 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     using Cfg = FwdCfg<D>;
     constexpr int S = Cfg::kStages;
 
-    const int bh = blockIdx.x;
+    // Launch order: the (sequence, query head) pairs are taken in chunks of p.head_chunk; inside a chunk the
+    // CTAs go query-tile pair by pair (heaviest first), chunk after chunk, so the K/V rows that the CTAs
+    // running at one time walk through fit the L2 (the host picks the chunk from the K/V size per head).
+    const int bh = (int)blockIdx.y * p.head_chunk + (int)blockIdx.x % p.head_chunk;
+    if (bh >= p.B * p.Hq) return;
+    const int pair_raw = (int)blockIdx.x / p.head_chunk;
+    const int n_pairs_grid = (int)gridDim.x / p.head_chunk;
     const int b = bh / p.Hq, h = bh % p.Hq;
     const int g = h / (p.Hq / p.Hkv);
-    const int pair = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest (latest) query tiles first
+    const int pair = n_pairs_grid - 1 - pair_raw;  // heaviest (latest) query tiles first
     const int r0 = p.cu_seqlens[b];
     const int r1 = p.cu_seqlens[b + 1];
     int L = r1 - r0;

@@ -4,6 +4,7 @@
 #include "../../include/sdpa.h"
 
 #include <math.h>
+#include <algorithm>
 #include <mutex>
 
 #include "bwd_kernel.cuh"
@@ -121,6 +122,21 @@ static int check_common(const int32_t* cu, int B, int Hq, int Hkv, int D, float 
     return SDPA_OK;
 }
 
+// Forward launch order: how many (sequence, query head) pairs have their CTAs interleaved.  When all K/V
+// rows fit the L2 comfortably every pair is interleaved (heaviest query tiles of all heads first, the best
+// balance); otherwise a chunk covers as many kv heads as keep about 48 MB of K/V in flight, so that the
+// query tiles of one head re-read its K/V from the L2 instead of from DRAM.
+static int fwd_head_chunk(int B, int Hq, int Hkv, int D, long long kv_rows) {
+    const long long kL2Budget = 48ll << 20;
+    const long long total = kv_rows * Hkv * D * 4;  // K and V, bf16
+    const int all = B * Hq;
+    if (total <= kL2Budget || B <= 0) return all;
+    const long long per_kv_head = std::max<long long>(1, kv_rows / B * D * 4);
+    const long long kv_heads = std::max<long long>(1, kL2Budget / per_kv_head);
+    const long long chunk = kv_heads * (Hq / Hkv);
+    return static_cast<int>(std::min<long long>(all, chunk));
+}
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static size_t bwd_dq_bytes(int Hq, int D, int T) { return align_up(static_cast<size_t>(T) * Hq * D * sizeof(float), 256); }
 static size_t bwd_delta_bytes(int Hq, int T) { return align_up(static_cast<size_t>(T) * Hq * sizeof(float), 256); }
@@ -160,7 +176,10 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
     p.scale_log2 = scale * 1.4426950408889634f;
     const int n_pairs = (max_seqlen + 255) / 256;
     if (n_pairs > 65535) return SDPA_ERR_SHAPE;
-    dim3 grid(static_cast<unsigned>(B * Hq), static_cast<unsigned>(n_pairs), 1);
+    p.head_chunk = fwd_head_chunk(B, Hq, Hkv, D, total_tokens);
+    if (static_cast<long long>(n_pairs) * p.head_chunk > 0x7fffffffLL) return SDPA_ERR_SHAPE;
+    dim3 grid(static_cast<unsigned>(n_pairs * p.head_chunk),
+              static_cast<unsigned>((B * Hq + p.head_chunk - 1) / p.head_chunk), 1);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (D == 128)
         sdpa_fwd_kernel<128, false><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, p);
@@ -205,7 +224,10 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
     p.scale_log2 = scale * 1.4426950408889634f;
     const int n_pairs = (max_seqlen_q + 255) / 256;
     if (n_pairs > 65535) return SDPA_ERR_SHAPE;
-    dim3 grid(static_cast<unsigned>(B * Hq), static_cast<unsigned>(n_pairs), 1);
+    p.head_chunk = fwd_head_chunk(B, Hq, Hkv, D, num_pages);
+    if (static_cast<long long>(n_pairs) * p.head_chunk > 0x7fffffffLL) return SDPA_ERR_SHAPE;
+    dim3 grid(static_cast<unsigned>(n_pairs * p.head_chunk),
+              static_cast<unsigned>((B * Hq + p.head_chunk - 1) / p.head_chunk), 1);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the K/V tensor maps are unused by the gathering producer; the Q map stands in for them
     if (D == 128)
