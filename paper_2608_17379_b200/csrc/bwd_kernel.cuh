@@ -30,17 +30,12 @@ namespace sdpa {
 __device__ long long g_trace[5 * 32 * 8];
 #define SDPA_TR(role, it, k)                                                                   \
     do {                                                                                       \
-        if (blockIdx.y == 0 && blockIdx.x == 4 * SDPA_BWD_GROUP_CHUNK && (it) >= 8 && (it) < 40)                       \
+        if (blockIdx.y == 0 && blockIdx.x == 4 * 8 && (it) >= 8 && (it) < 40)                       \
             g_trace[((role) * 32 + ((it) - 8)) * 8 + (k)] = clock64();                         \
     } while (0)
 #else
 #define SDPA_TR(role, it, k) do { } while (0)
 #endif
-
-#ifndef SDPA_BWD_GROUP_CHUNK
-#define SDPA_BWD_GROUP_CHUNK 8
-#endif
-constexpr int kBwdGroupChunk = SDPA_BWD_GROUP_CHUNK;  // (sequence, kv head) groups whose CTAs are launched interleaved
 
 struct BwdParams {
     const int32_t* cu_seqlens;
@@ -53,6 +48,7 @@ struct BwdParams {
     int B, Hq, Hkv, T;
     int causal;
     int max_seqlen;
+    int group_chunk;  // (sequence, kv head) groups whose CTAs are launched interleaved
     float scale;
     float scale_log2;
 };
@@ -145,13 +141,13 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const BwdParams p) {
     using Cfg = BwdCfg<D>;
     constexpr int NS = Cfg::kQStages;
-    // Launch order: the (sequence, kv head) groups are taken in chunks of kBwdGroupChunk; inside a chunk the
+    // Launch order: the (sequence, kv head) groups are taken in chunks of p.group_chunk; inside a chunk the
     // CTAs go key tile by key tile (under a causal mask the low key tiles see the most queries, so the heavy
     // CTAs start first), chunk after chunk.  CTAs that run at the same time therefore belong to few groups
     // and sweep the same query heads at about the same time, which keeps the part of the fp32 dQ accumulator
     // being reduced into inside the L2; one chunk for everything would spread a wave over all groups and
     // every accumulator line would travel to DRAM and back once per wave.
-    const int bg = static_cast<int>(blockIdx.y) * kBwdGroupChunk + static_cast<int>(blockIdx.x) % kBwdGroupChunk;
+    const int bg = static_cast<int>(blockIdx.y) * p.group_chunk + static_cast<int>(blockIdx.x) % p.group_chunk;
     if (bg >= p.B * p.Hkv) return;
     const int b = bg / p.Hkv, g = bg % p.Hkv;
     const int G = p.Hq / p.Hkv;
@@ -163,8 +159,8 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         return;
     }
     // causal: low key tiles see the most query tiles -> launch them first
-    const int n_tiles_grid = static_cast<int>(gridDim.x) / kBwdGroupChunk;
-    const int jt_raw = static_cast<int>(blockIdx.x) / kBwdGroupChunk;
+    const int n_tiles_grid = static_cast<int>(gridDim.x) / p.group_chunk;
+    const int jt_raw = static_cast<int>(blockIdx.x) / p.group_chunk;
     const int jt = p.causal ? jt_raw : n_tiles_grid - 1 - jt_raw;
     const int kv0 = jt * 128;
     if (kv0 >= L) return;

@@ -137,6 +137,17 @@ static int fwd_head_chunk(int B, int Hq, int Hkv, int D, long long kv_rows) {
     return static_cast<int>(std::min<long long>(all, chunk));
 }
 
+// Backward launch order: how many (sequence, kv head) groups have their CTAs interleaved.  A small dQ
+// accumulator stays in the L2 whatever the order, so all groups are interleaved (heaviest key tiles first).
+// Otherwise a chunk holds about two waves of CTAs (at least 8 groups), in equal chunks: the CTAs running
+// at one time then reduce into few heads' accumulator rows, which stay in the L2 between their visits.
+static int bwd_group_chunk(int n_groups, int n_kv_tiles, long long dq_acc_bytes) {
+    if (dq_acc_bytes <= (48ll << 20) || n_groups <= 8) return std::max(1, n_groups);
+    const int c0 = std::max(8, (296 + n_kv_tiles - 1) / std::max(1, n_kv_tiles));
+    const int n_chunks = (n_groups + c0 - 1) / c0;
+    return (n_groups + n_chunks - 1) / n_chunks;
+}
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static size_t bwd_dq_bytes(int Hq, int D, int T) { return align_up(static_cast<size_t>(T) * Hq * D * sizeof(float), 256); }
 static size_t bwd_delta_bytes(int Hq, int T) { return align_up(static_cast<size_t>(T) * Hq * sizeof(float), 256); }
@@ -304,10 +315,12 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
     p.scale_log2 = scale * 1.4426950408889634f;
     const int n_kv_tiles = (max_seqlen + 127) / 128;
     if (n_kv_tiles > 65535) return SDPA_ERR_SHAPE;
-    // x walks a chunk of kGroupChunk (sequence, kv head) groups key tile by key tile, y walks the chunks
+    // x walks a chunk of (sequence, kv head) groups key tile by key tile, y walks the chunks
     const int n_groups = B * Hkv;
-    dim3 grid(static_cast<unsigned>(n_kv_tiles * sdpa::kBwdGroupChunk),
-              static_cast<unsigned>((n_groups + sdpa::kBwdGroupChunk - 1) / sdpa::kBwdGroupChunk), 1);
+    p.group_chunk = bwd_group_chunk(n_groups, n_kv_tiles, static_cast<long long>(total_tokens) * Hq * D * 4);
+    if (static_cast<long long>(n_kv_tiles) * p.group_chunk > 0x7fffffffLL) return SDPA_ERR_SHAPE;
+    dim3 grid(static_cast<unsigned>(n_kv_tiles * p.group_chunk),
+              static_cast<unsigned>((n_groups + p.group_chunk - 1) / p.group_chunk), 1);
     if (tl_ev_main_start) SDPA_CUDA_TRY(cudaEventRecord(tl_ev_main_start, s));
     if (D == 128)
         sdpa_bwd_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
