@@ -32,7 +32,7 @@ METRIC = "SDPA fwd+bwd TFLOPS (bf16, device-timed)"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this same command on
 # the c3 workload (profiles/sdpa_kernels_c3_dram.md); null for other workloads.
-NCU_DRAM_TRAFFIC_C3 = {"sdpa_bwd_kernel<128>": 648844288 + 308653056, "sdpa_fwd_kernel<128>": 100847616 + 35015168}
+NCU_DRAM_TRAFFIC_C3 = {"sdpa_bwd_kernel<128>": 365212928 + 155866112, "sdpa_fwd_kernel<128>": 101782784 + 36194304}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
