@@ -22,8 +22,10 @@
  *  - Grouped-query attention: query head h reads kv head h / (Hq / Hkv).
  *  - causal != 0: query i of a sequence attends to keys 0..i of that sequence
  *    (lower-triangular mask); causal == 0: to all keys of its sequence.
- *  - Supported: D in {64, 128}; Hq a multiple of Hkv; scale finite and > 0; sequences of any
- *    length >= 0 (empty sequences and T = 0 are valid no-ops).
+ *  - Supported: D a multiple of 8 with 8 <= D <= 128 (the kernels are built for 64 and 128; another D
+ *    runs in the next larger one with zero-padded columns, e.g. the paper's head dimension 96 at 3/4 of
+ *    the arithmetic efficiency of 128; appendix "Workloads"); Hq a multiple of Hkv; scale finite and
+ *    > 0; sequences of any length >= 0 (empty sequences and T = 0 are valid no-ops).
  *  - max_seqlen must be >= the longest sequence; total_tokens must equal cu_seqlens[B].  They
  *    size the launch grid and the TMA tensor maps without a device-to-host read of cu_seqlens.
  *    A cu_seqlens that contradicts them is reported through sdpa_query_status

@@ -41,13 +41,14 @@ struct BwdParams {
     const int32_t* cu_seqlens;
     const float* lse;    // [Hq, T]
     const float* delta;  // [Hq, T]
-    float* dq_acc;       // [Hq, T, D] fp32 (head-major)
+    float* dq_acc;       // [Hq, T, D] fp32 (head-major; D = the kernel's padded head dimension)
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     int* status;
     int B, Hq, Hkv, T;
     int causal;
     int max_seqlen;
+    int d;            // head dimension of the tensors (multiple of 8, <= D of the kernel; the rest is zero padding)
     int group_chunk;  // (sequence, kv head) groups whose CTAs are launched interleaved
     float scale;
     float scale_log2;
@@ -83,7 +84,7 @@ enum BwdSite {
 template <int D>
 __global__ void __launch_bounds__(256)
 sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ dout,
-                           float* __restrict__ delta, float* __restrict__ dq_acc, int T, int Hq) {
+                           float* __restrict__ delta, float* __restrict__ dq_acc, int T, int Hq, int d) {
     constexpr int kLanesPerRow = D / 8;
     const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     const long long row = gid / kLanesPerRow;  // row = token * Hq + head
@@ -91,8 +92,11 @@ sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloa
     const long long rows = static_cast<long long>(T) * Hq;
     float acc = 0.f;
     if (row < rows) {
-        const uint4 a = *reinterpret_cast<const uint4*>(o + row * D + part * 8);
-        const uint4 b = *reinterpret_cast<const uint4*>(dout + row * D + part * 8);
+        uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;  // padding columns d..D-1 contribute nothing
+        if (part * 8 < d) {
+            a = *reinterpret_cast<const uint4*>(o + row * d + part * 8);
+            b = *reinterpret_cast<const uint4*>(dout + row * d + part * 8);
+        }
         const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
         const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
@@ -115,10 +119,10 @@ sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloa
 
 __global__ void __launch_bounds__(256)
 sdpa_bwd_dq_convert_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq, long long n8, float scale,
-                           int T, int Hq, int D) {
+                           int T, int Hq, int D, int d) {
     const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;  // output group of 8
     if (i >= n8) return;
-    const int d8 = D / 8;
+    const int d8 = d / 8;  // output rows have d columns, accumulator rows D (padded)
     const int part = static_cast<int>(i % d8);
     const long long th = i / d8;
     const int h = static_cast<int>(th % Hq);
@@ -380,9 +384,9 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                 for (int pass = 0; pass < 32 / kRowsPerPass; ++pass) {
                     const int rr = (warp & 3) * 32 + pass * kRowsPerPass + lane / kChunks;
-                    if (rr < rows_left) {
+                    if (rr < rows_left && k * 8 < p.d) {
                         const uint4 w = *reinterpret_cast<const uint4*>(out_stage + rr * (D * 2) + ((k ^ (rr & 7)) << 4));
-                        __nv_bfloat16* dst = out + (static_cast<size_t>(r0 + kv0 + rr) * p.Hkv + g) * D;
+                        __nv_bfloat16* dst = out + (static_cast<size_t>(r0 + kv0 + rr) * p.Hkv + g) * p.d;
                         *reinterpret_cast<uint4*>(dst + k * 8) = w;
                     }
                 }

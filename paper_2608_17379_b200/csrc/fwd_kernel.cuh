@@ -37,6 +37,7 @@ struct FwdParams {
     int B, Hq, Hkv, T;
     int causal;
     int max_seqlen;
+    int d;             // head dimension of the tensors (multiple of 8, <= D of the kernel; columns d..D-1 are zero padding)
     int head_chunk;    // (sequence, query head) pairs whose CTAs are launched interleaved
     float scale;       // softmax scale
     float scale_log2;  // scale * log2(e)
@@ -325,9 +326,9 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                 for (int pass = 0; pass < 32 / kRowsPerPass; ++pass) {
                     const int rr = (warp & 3) * 32 + pass * kRowsPerPass + lane / kChunks;  // row inside the tile
-                    if (rr < rows_left) {
+                    if (rr < rows_left && k * 8 < p.d) {
                         const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * (D * 2) + ((k ^ (rr & 7)) << 4));
-                        __nv_bfloat16* dst = p.o + (static_cast<size_t>(r0 + q_start + t * 128 + rr) * p.Hq + h) * D;
+                        __nv_bfloat16* dst = p.o + (static_cast<size_t>(r0 + q_start + t * 128 + rr) * p.Hq + h) * p.d;
                         *reinterpret_cast<uint4*>(dst + k * 8) = w;
                     }
                 }
@@ -382,11 +383,13 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     for (int i = 0; i < 4; ++i) {
                         const int row = lane + 32 * i;
                         const bool have = page[i] >= 0;
-                        const __nv_bfloat16* src = cache + (static_cast<size_t>(have ? page[i] : 0) * p.Hkv + g) * D;
+                        const __nv_bfloat16* src = cache + (static_cast<size_t>(have ? page[i] : 0) * p.Hkv + g) * p.d;
 #pragma unroll
-                        for (int c = 0; c < D / 8; ++c)
-                            cp_async_16(dst + (c >> 3) * Cfg::kAtomBytes + sw128_offset(row, c & 7), src + c * 8,
-                                        have ? 16u : 0u);
+                        for (int c = 0; c < D / 8; ++c) {
+                            const bool real = have && c * 8 < p.d;  // padding columns and missing rows are zero-filled
+                            cp_async_16(dst + (c >> 3) * Cfg::kAtomBytes + sw128_offset(row, c & 7), real ? src + c * 8 : src,
+                                        real ? 16u : 0u);
+                        }
                     }
                     cp_async_commit();
                     if (pending >= 0) {

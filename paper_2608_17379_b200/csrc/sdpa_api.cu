@@ -109,12 +109,16 @@ static int make_map(CUtensorMap* map, const void* base, int T, int H, int D, int
     return SDPA_OK;
 }
 
+// Head dimension the kernels are instantiated for: 64 or 128; a smaller head dimension runs in the next
+// larger kernel, its missing columns zero-filled by the TMA loads (out-of-bounds box columns read as 0).
+static int padded_head_dim(int D) { return D <= 64 ? 64 : 128; }
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int check_common(const int32_t* cu, int B, int Hq, int Hkv, int D, float scale, int T, int max_seqlen) {
     if (cu == nullptr) return SDPA_ERR_NULL;
     if (B < 1 || Hq < 1 || Hkv < 1 || T < 0 || max_seqlen < 0) return SDPA_ERR_SHAPE;
-    if (D != 64 && D != 128) return SDPA_ERR_SHAPE;
+    if (D < 8 || D > 128 || (D % 8) != 0) return SDPA_ERR_SHAPE;
     if (Hq % Hkv != 0) return SDPA_ERR_SHAPE;
     if (!(scale > 0.f) || !isfinite(scale)) return SDPA_ERR_SHAPE;
     if (max_seqlen > T) return SDPA_ERR_SHAPE;
@@ -183,6 +187,7 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.T = total_tokens;
     p.causal = causal ? 1 : 0;
     p.max_seqlen = max_seqlen;
+    p.d = D;
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
     const int n_pairs = (max_seqlen + 255) / 256;
@@ -192,7 +197,7 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
     dim3 grid(static_cast<unsigned>(n_pairs * p.head_chunk),
               static_cast<unsigned>((B * Hq + p.head_chunk - 1) / p.head_chunk), 1);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (D == 128)
+    if (padded_head_dim(D) == 128)
         sdpa_fwd_kernel<128, false><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, p);
     else
         sdpa_fwd_kernel<64, false><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mk, mv, p);
@@ -231,6 +236,7 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.T = total_q;
     p.causal = causal ? 1 : 0;
     p.max_seqlen = max_seqlen_q;
+    p.d = D;
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
     const int n_pairs = (max_seqlen_q + 255) / 256;
@@ -241,7 +247,7 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
               static_cast<unsigned>((B * Hq + p.head_chunk - 1) / p.head_chunk), 1);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the K/V tensor maps are unused by the gathering producer; the Q map stands in for them
-    if (D == 128)
+    if (padded_head_dim(D) == 128)
         sdpa_fwd_kernel<128, true><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mq, mq, p);
     else
         sdpa_fwd_kernel<64, true><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mq, mq, p);
@@ -250,9 +256,9 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
 }
 
 extern "C" size_t sdpa_bwd_workspace_bytes(int B, int Hq, int Hkv, int D, int total_tokens, int max_seqlen) {
-    if (B < 1 || Hq < 1 || Hkv < 1 || total_tokens < 0 || max_seqlen < 0 || (D != 64 && D != 128) || Hq % Hkv != 0)
+    if (B < 1 || Hq < 1 || Hkv < 1 || total_tokens < 0 || max_seqlen < 0 || D < 8 || D > 128 || (D % 8) != 0 || Hq % Hkv != 0)
         return 0;
-    return bwd_dq_bytes(Hq, D, total_tokens) + bwd_delta_bytes(Hq, total_tokens) + 256;
+    return bwd_dq_bytes(Hq, padded_head_dim(D), total_tokens) + bwd_delta_bytes(Hq, total_tokens) + 256;
 }
 
 extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
@@ -275,22 +281,23 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
     float* dq_acc = static_cast<float*>(workspace);
-    float* delta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + bwd_dq_bytes(Hq, D, total_tokens));
+    const int Dp = padded_head_dim(D);
+    float* delta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + bwd_dq_bytes(Hq, Dp, total_tokens));
 
     // B0: D_i = rowsum(dO * O), and clear the fp32 dQ accumulator.
     {
         const long long rows = static_cast<long long>(total_tokens) * Hq;
         const int threads = 256;
-        const int rows_per_block = threads / (D / 8);
+        const int rows_per_block = threads / (Dp / 8);
         const long long blocks = (rows + rows_per_block - 1) / rows_per_block;
-        if (D == 128)
+        if (Dp == 128)
             sdpa_bwd_preprocess_kernel<128><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
                 static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
-                total_tokens, Hq);
+                total_tokens, Hq, D);
         else
             sdpa_bwd_preprocess_kernel<64><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
                 static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
-                total_tokens, Hq);
+                total_tokens, Hq, D);
         SDPA_CUDA_TRY(cudaGetLastError());
     }
 
@@ -317,12 +324,13 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
     if (n_kv_tiles > 65535) return SDPA_ERR_SHAPE;
     // x walks a chunk of (sequence, kv head) groups key tile by key tile, y walks the chunks
     const int n_groups = B * Hkv;
-    p.group_chunk = bwd_group_chunk(n_groups, n_kv_tiles, static_cast<long long>(total_tokens) * Hq * D * 4);
+    p.d = D;
+    p.group_chunk = bwd_group_chunk(n_groups, n_kv_tiles, static_cast<long long>(total_tokens) * Hq * Dp * 4);
     if (static_cast<long long>(n_kv_tiles) * p.group_chunk > 0x7fffffffLL) return SDPA_ERR_SHAPE;
     dim3 grid(static_cast<unsigned>(n_kv_tiles * p.group_chunk),
               static_cast<unsigned>((n_groups + p.group_chunk - 1) / p.group_chunk), 1);
     if (tl_ev_main_start) SDPA_CUDA_TRY(cudaEventRecord(tl_ev_main_start, s));
-    if (D == 128)
+    if (Dp == 128)
         sdpa_bwd_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
     else
         sdpa_bwd_kernel<64><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, s>>>(mq, mk, mv, mdo, p);
@@ -335,7 +343,7 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
         const int threads = 256;
         const long long blocks = (n8 + threads - 1) / threads;
         sdpa_bwd_dq_convert_kernel<<<static_cast<unsigned>(blocks), threads, 0, s>>>(
-            dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale, total_tokens, Hq, D);
+            dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale, total_tokens, Hq, Dp, D);
         SDPA_CUDA_TRY(cudaGetLastError());
     }
     return SDPA_OK;

@@ -165,17 +165,19 @@ def config(name: str) -> Workload:
         lens = tuple(int(x) for x in gen_lengths(4, 8, 512, 8192))
         return Workload("c5", 4, lens, 32, 4, 128, True)
     # The paper's own primary attention shape (appendix "Workloads": batch 4, 48 heads, sequence 4096)
-    # and its d64 generalisation shape; context workloads, not part of the five benchmark configs.
+    # and its d64 / d96 generalisation shapes; context workloads, not part of the five benchmark configs.
     if name == "mha":
         return Workload("mha", 5, (4096,) * 4, 48, 48, 128, False)
     if name == "mha_causal":
         return Workload("mha_causal", 5, (4096,) * 4, 48, 48, 128, True)
     if name == "mha_d64":
         return Workload("mha_d64", 6, (4096,) * 4, 48, 48, 64, True)
+    if name == "mha_d96":
+        return Workload("mha_d96", 7, (4096,) * 4, 48, 48, 96, True)
     raise KeyError(name)
 
 
-CONFIG_NAMES = ("c1", "c2", "c3", "c4", "c4c", "c5", "mha", "mha_causal", "mha_d64")
+CONFIG_NAMES = ("c1", "c2", "c3", "c4", "c4c", "c5", "mha", "mha_causal", "mha_d64", "mha_d96")
 
 
 def make_inputs(w: Workload):

@@ -47,14 +47,18 @@ def test_argument_checks_come_before_any_cuda_call(lib):
     assert fwd(cu=None) == -1
     assert fwd(q=None) == -1
     assert fwd(q=a + 2) == -2
-    assert fwd(D=96) == -3
+    assert fwd(D=100) == -3   # not a multiple of 8
+    assert fwd(D=136) == -3   # above the largest kernel
+    assert fwd(D=0) == -3
     assert fwd(Hq=3, Hkv=2) == -3
     assert fwd(B=0) == -3
     assert fwd(scale=0.0) == -3
     assert fwd(scale=float("nan")) == -3
     assert fwd(L=9, T=8) == -3
     assert fwd(T=0, L=0) == 0  # empty batch: valid no-op
-    assert lib.sdpa_bwd_workspace_bytes(1, 2, 2, 96, 8, 8) == 0
+    assert lib.sdpa_bwd_workspace_bytes(1, 2, 2, 100, 8, 8) == 0
+    # head dimension 96 runs in the 128-wide kernel: the fp32 dQ accumulator is padded to 128 columns
+    assert lib.sdpa_bwd_workspace_bytes(1, 2, 2, 96, 8, 8) == lib.sdpa_bwd_workspace_bytes(1, 2, 2, 128, 8, 8)
     need = lib.sdpa_bwd_workspace_bytes(1, 2, 2, 64, 8, 8)
     assert need >= 8 * 2 * 64 * 4 + 8 * 2 * 4
     bwd = lambda ws, n: lib.sdpa_bwd(a, a, a, a, a, a, a, a, a, a, 1, 2, 2, 64, 0, 1.0, 8, 8, ws, n, None)

@@ -37,6 +37,8 @@ def _run(q_lens, k_lens, Hq, Hkv, D, num_pages, causal, seed):
     ((130,), (130,), 2, 2, 128),
     ((300, 77), (300, 77), 4, 2, 128),
     ((100, 1, 257), (400, 130, 257), 6, 2, 128),   # more keys than queries: end-aligned causal mask
+    ((90, 200), (300, 200), 4, 2, 96),             # head dimension between the kernels: zero-padded columns
+    ((33,), (140,), 2, 1, 40),
 ])
 def test_small_paged_shapes(q_lens, k_lens, Hq, Hkv, D, causal):
     _run(q_lens, k_lens, Hq, Hkv, D, num_pages=int(sum(k_lens)) + 37, causal=causal, seed=300 + len(q_lens) + Hq)

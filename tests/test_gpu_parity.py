@@ -76,7 +76,7 @@ def test_paper_ragged_shape():
 
 
 # ------------------------------------------------------------------ full-size configurations, sampled slices
-@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c4c", "c5", "mha", "mha_causal", "mha_d64"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c4c", "c5", "mha", "mha_causal", "mha_d64", "mha_d96"])
 def test_full_configs_on_sampled_slices(name):
     """The five benchmark configurations in the launch configuration the bench times; the oracle
     checks complete O/LSE/dQ/dK/dV of independent (sequence, kv-head) slices."""
@@ -268,7 +268,7 @@ def test_host_buffer_entry_point_matches_device_entry_points():
 
 # ------------------------------------------------------------------ randomised shapes
 def test_random_shapes_against_the_oracle():
-    """Thirty random small problems (ragged lengths incl. zeros, MHA/GQA, both head dims, both masks)."""
+    """Thirty random small problems (ragged lengths incl. zeros, MHA/GQA, several head dims, both masks)."""
     rng = np.random.default_rng(2024)
     for case in range(30):
         B = int(rng.integers(1, 5))
@@ -277,7 +277,24 @@ def test_random_shapes_against_the_oracle():
             lengths[0] = 17
         Hkv = int(rng.choice([1, 2, 3]))
         G = int(rng.choice([1, 2, 4]))
-        D = int(rng.choice([64, 128]))
+        D = int(rng.choice([64, 128, 128, 96, 32]))
         causal = bool(rng.integers(0, 2))
         w = TL.random_workload(lengths, Hkv * G, Hkv, D, causal, seed=5000 + case, qk_mul=float(rng.choice([1.0, 2.0])))
         run_and_compare(w)
+
+
+# ------------------------------------------------------------------ head dimensions between the kernels
+@pytest.mark.parametrize("D", [8, 24, 72, 96, 120])
+@pytest.mark.parametrize("causal", [False, True])
+def test_head_dims_that_run_zero_padded(D, causal):
+    """Head dimensions other than 64 / 128 run in the next larger kernel with zero-padded columns
+    (appendix "Workloads" lists head dimension 96); outputs must not depend on the padding."""
+    w = TL.random_workload((300, 129, 64), 4, 2, D, causal, seed=7100 + D)
+    run_and_compare(w)
+
+
+def test_d96_paper_shape_slices():
+    """The paper's d96 generalisation shape (batch 4, 48 heads, sequence 4096), reduced to one sequence
+    and 8 heads so that the oracle checks every slice in seconds."""
+    w = TL.random_workload((4096,), 8, 8, 96, True, seed=7196)
+    run_and_compare(w, slices=[(0, 0), (0, 7)])
