@@ -84,7 +84,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.003)
 
     def __enter__(self):
         if self.nv is not None:
@@ -314,8 +314,6 @@ def main():
         torch.cuda.synchronize()
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    ev_ms, ev_me = ev(), ev()
-    ev_ms.record(); ev_me.record()  # create the underlying CUDA events
     for _ in range(args.warmup):
         fwd(); bwd()
     barrier()
@@ -323,23 +321,24 @@ def main():
 
     K = args.steps
     e_f0 = [ev() for _ in range(K)]; e_f1 = [ev() for _ in range(K)]; e_b1 = [ev() for _ in range(K)]
-    main_ms = []
-    binding.bwd_profile_events(ev_ms, ev_me)
+    # the main backward kernel is bracketed by its own pair of events in every timed step (the library
+    # records them around that launch), so its duration is measured inside the timed region
+    e_m0 = [ev() for _ in range(K)]; e_m1 = [ev() for _ in range(K)]
+    for a, b in zip(e_m0, e_m1):
+        a.record(); b.record()  # create the underlying CUDA events
     with ClockSampler(local_rank) as clocks:
         barrier()
         t_start, t_stop = ev(), ev()
         t_start.record()
         for i in range(K):
-            e_f0[i].record(); fwd(); e_f1[i].record(); bwd(); e_b1[i].record()
+            e_f0[i].record(); fwd(); e_f1[i].record()
+            binding.bwd_profile_events(e_m0[i], e_m1[i])
+            bwd(); e_b1[i].record()
         t_stop.record()
         barrier()
     total_ms = t_start.elapsed_time(t_stop)
     binding.bwd_profile_events(None, None)
-    # main backward kernel alone: a few extra launches with the profiling events read back each time
-    binding.bwd_profile_events(ev_ms, ev_me)
-    for _ in range(min(K, 20)):
-        bwd(); torch.cuda.synchronize(); main_ms.append(ev_ms.elapsed_time(ev_me))
-    binding.bwd_profile_events(None, None)
+    main_ms = [e_m0[i].elapsed_time(e_m1[i]) for i in range(K)]
     status = binding.query_status()
     assert status == (0, 0), status
 

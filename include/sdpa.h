@@ -117,6 +117,29 @@ int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same forward and backward passes on dense tensors in the shape convention of the paper's attention
+ * workloads (appendix "Workloads": bf16 tensors of shape [batch, heads, sequence, head dim]):
+ *        q, o, dout, dq : bf16 [B, Hq,  S, D]      k, v, dk, dv : bf16 [B, Hkv, S, D]
+ *        lse            : fp32 [B, Hq, S]
+ * all contiguous.  cu_seqlens may be null: every sequence then has S rows.  Otherwise it is the usual
+ * int32 [B + 1] device array and sequence b uses rows 0 .. cu_seqlens[b+1] - cu_seqlens[b] - 1 (at most S)
+ * of its [H, S, D] blocks.  Rows past a sequence's length never influence a result, but the tile loads
+ * read them and multiply them by zero weights, so they must hold finite values (zeros, or anything left
+ * by an earlier finite computation); in o, lse, dk and dv such rows are left untouched, in dq they are
+ * written as zeros.  No transposed copy is made: the TMA tensor maps and the
+ * stores walk the dense layout directly.  The backward workspace is sized by
+ * sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, B * S, S).  B * S must fit a 32-bit integer.  Everything else
+ * (masking, GQA mapping, supported D, errors, status word) is as for sdpa_fwd / sdpa_bwd.
+ */
+int sdpa_fwd_bhsd(const void* q, const void* k, const void* v, void* o, float* lse,
+                  const int32_t* cu_seqlens, int B, int Hq, int Hkv, int S, int D, int causal,
+                  float scale, void* stream);
+int sdpa_bwd_bhsd(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                  const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B,
+                  int Hq, int Hkv, int S, int D, int causal, float scale, void* workspace,
+                  size_t workspace_bytes, void* stream);
+
+/*
  * Backward pass for callers that may not allocate device memory (the paper has no counterpart: this
  * is a convenience of this library, not one of its operators).
  *

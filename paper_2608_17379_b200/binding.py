@@ -18,7 +18,8 @@ _LIB = None
 SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
-           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout", "sdpa_fwd_paged")
+           "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout", "sdpa_fwd_paged",
+           "sdpa_fwd_bhsd", "sdpa_bwd_bhsd")
 
 
 class SdpaError(RuntimeError):
@@ -53,6 +54,10 @@ def load():
     lib.sdpa_selftest_wait_timeout.argtypes = [ctypes.c_longlong, vp]
     lib.sdpa_fwd_paged.restype = ci
     lib.sdpa_fwd_paged.argtypes = [vp] * 8 + [ci, ci, ci, ci, ci, cf, ci, ci, ci, vp]
+    lib.sdpa_fwd_bhsd.restype = ci
+    lib.sdpa_fwd_bhsd.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp]
+    lib.sdpa_bwd_bhsd.restype = ci
+    lib.sdpa_bwd_bhsd.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
     lib.gemm_bf16_nt.restype = ci
     lib.gemm_bf16_nt.argtypes = [vp, vp, vp, ci, ci, ci, vp]
     lib.sdpa_query_status.restype = ci
@@ -133,6 +138,48 @@ def sdpa_bwd(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, s
                       _ptr(cu_seqlens), B, Hq, Hkv, D, int(bool(causal)), float(scale), T, int(max_seqlen),
                       _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
     _check(rc, "sdpa_bwd")
+    return dq, dk, dv
+
+
+def _dims_bhsd(q, k):
+    assert q.dim() == 4 and k.dim() == 4 and q.is_contiguous() and k.is_contiguous()
+    assert q.dtype == torch.bfloat16 and k.dtype == torch.bfloat16 and q.is_cuda and k.is_cuda
+    B, Hq, S, D = q.shape
+    assert k.shape[0] == B and k.shape[2] == S and k.shape[3] == D
+    return B, Hq, k.shape[1], S, D
+
+
+def sdpa_fwd_bhsd(q, k, v, causal: bool, scale: float, cu_seqlens=None, o=None, lse=None, stream=None):
+    """Dense layout: q [B,Hq,S,D], k,v [B,Hkv,S,D] bf16 contiguous; cu_seqlens (optional int32 [B+1] on the
+    device) gives per-sequence lengths <= S.  Returns (o [B,Hq,S,D] bf16, lse [B,Hq,S] fp32)."""
+    lib = load()
+    B, Hq, Hkv, S, D = _dims_bhsd(q, k)
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
+    rc = lib.sdpa_fwd_bhsd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(cu_seqlens) if cu_seqlens is not None else None,
+                           B, Hq, Hkv, S, D, int(bool(causal)), float(scale), _stream_ptr(stream))
+    _check(rc, "sdpa_fwd_bhsd")
+    return o, lse
+
+
+def sdpa_bwd_bhsd(q, k, v, o, lse, dout, causal: bool, scale: float, cu_seqlens=None, dq=None, dk=None, dv=None,
+                  workspace=None, stream=None):
+    """Gradients for the dense layout; tensors as in sdpa_fwd_bhsd."""
+    lib = load()
+    B, Hq, Hkv, S, D = _dims_bhsd(q, k)
+    need = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, B * S, S)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    rc = lib.sdpa_bwd_bhsd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
+                           _ptr(cu_seqlens) if cu_seqlens is not None else None, B, Hq, Hkv, S, D,
+                           int(bool(causal)), float(scale), _ptr(workspace), int(workspace.numel()),
+                           _stream_ptr(stream))
+    _check(rc, "sdpa_bwd_bhsd")
     return dq, dk, dv
 
 

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libsdpa_b200.so")
 SOURCES = [os.path.join(CSRC, "sdpa_api.cu")]
-HEADERS = [os.path.join(CSRC, f) for f in ("ptx.cuh", "fwd_kernel.cuh", "bwd_kernel.cuh", "gemm_kernel.cuh")] + [
+HEADERS = [os.path.join(CSRC, f) for f in ("ptx.cuh", "layout.cuh", "fwd_kernel.cuh", "bwd_kernel.cuh", "gemm_kernel.cuh")] + [
     os.path.join(os.path.dirname(HERE), "include", "sdpa.h")]
 
 

@@ -23,6 +23,7 @@
 // compute groups have read it); the dS^T buffer is reused after ds_free (both dK and dQ^T finished).
 #pragma once
 #include "ptx.cuh"
+#include "layout.cuh"
 
 namespace sdpa {
 
@@ -49,6 +50,7 @@ struct BwdParams {
     int causal;
     int max_seqlen;
     int d;            // head dimension of the tensors (multiple of 8, <= D of the kernel; the rest is zero padding)
+    TensorLayout lay;
     int group_chunk;  // (sequence, kv head) groups whose CTAs are launched interleaved
     float scale;
     float scale_log2;
@@ -84,18 +86,25 @@ enum BwdSite {
 template <int D>
 __global__ void __launch_bounds__(256)
 sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ dout,
-                           float* __restrict__ delta, float* __restrict__ dq_acc, int T, int Hq, int d) {
+                           float* __restrict__ delta, float* __restrict__ dq_acc, int T, int Hq, int d,
+                           const TensorLayout lay) {
     constexpr int kLanesPerRow = D / 8;
     const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const long long row = gid / kLanesPerRow;  // row = token * Hq + head
+    const long long row = gid / kLanesPerRow;  // row = global token * Hq + head
     const int part = static_cast<int>(gid % kLanesPerRow);
     const long long rows = static_cast<long long>(T) * Hq;
     float acc = 0.f;
     if (row < rows) {
         uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;  // padding columns d..D-1 contribute nothing
         if (part * 8 < d) {
-            a = *reinterpret_cast<const uint4*>(o + row * d + part * 8);
-            b = *reinterpret_cast<const uint4*>(dout + row * d + part * 8);
+            long long off = row * d + part * 8;  // packed [T, Hq, d]: rows are contiguous
+            if (lay.dense) {
+                const int gt = static_cast<int>(row / Hq), hh = static_cast<int>(row % Hq);
+                off = (gt / lay.S) * lay.bs_q + static_cast<long long>(gt % lay.S) * lay.ts_q +
+                      static_cast<long long>(hh) * lay.hs_q + part * 8;
+            }
+            a = *reinterpret_cast<const uint4*>(o + off);
+            b = *reinterpret_cast<const uint4*>(dout + off);
         }
         const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
         const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
@@ -119,7 +128,7 @@ sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloa
 
 __global__ void __launch_bounds__(256)
 sdpa_bwd_dq_convert_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq, long long n8, float scale,
-                           int T, int Hq, int D, int d) {
+                           int T, int Hq, int D, int d, const TensorLayout lay) {
     const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;  // output group of 8
     if (i >= n8) return;
     const int d8 = d / 8;  // output rows have d columns, accumulator rows D (padded)
@@ -135,7 +144,13 @@ sdpa_bwd_dq_convert_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __re
     w.y = pack_bf16x2(a.z * scale, a.w * scale);
     w.z = pack_bf16x2(b.x * scale, b.y * scale);
     w.w = pack_bf16x2(b.z * scale, b.w * scale);
-    reinterpret_cast<uint4*>(dq)[i] = w;
+    long long off = i * 8;  // packed [T, Hq, d]: the output groups are contiguous
+    if (lay.dense) {
+        const int gt = static_cast<int>(t);
+        off = (gt / lay.S) * lay.bs_q + static_cast<long long>(gt % lay.S) * lay.ts_q +
+              static_cast<long long>(h) * lay.hs_q + part * 8;
+    }
+    *reinterpret_cast<uint4*>(dq + off) = w;
 }
 
 template <int D>
@@ -155,13 +170,13 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (bg >= p.B * p.Hkv) return;
     const int b = bg / p.Hkv, g = bg % p.Hkv;
     const int G = p.Hq / p.Hkv;
-    const int r0 = p.cu_seqlens[b];
-    const int r1 = p.cu_seqlens[b + 1];
-    const int L = r1 - r0;
-    if (L < 0 || r0 < 0 || r1 > p.T || L > p.max_seqlen) {
+    SeqPos sp;
+    if (!locate_sequence(p.lay, p.cu_seqlens, b, p.T, p.max_seqlen, sp)) {
         if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
         return;
     }
+    const int r0 = sp.tok0;  // token coordinate of the sequence's first row in the tensors
+    const int L = sp.L;
     // causal: low key tiles see the most query tiles -> launch them first
     const int n_tiles_grid = static_cast<int>(gridDim.x) / p.group_chunk;
     const int jt_raw = static_cast<int>(blockIdx.x) / p.group_chunk;
@@ -386,7 +401,9 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const int rr = (warp & 3) * 32 + pass * kRowsPerPass + lane / kChunks;
                     if (rr < rows_left && k * 8 < p.d) {
                         const uint4 w = *reinterpret_cast<const uint4*>(out_stage + rr * (D * 2) + ((k ^ (rr & 7)) << 4));
-                        __nv_bfloat16* dst = out + (static_cast<size_t>(r0 + kv0 + rr) * p.Hkv + g) * p.d;
+                        __nv_bfloat16* dst = out + sp.bidx * p.lay.bs_kv +
+                                             static_cast<long long>(r0 + kv0 + rr) * p.lay.ts_kv +
+                                             static_cast<long long>(g) * p.lay.hs_kv;
                         *reinterpret_cast<uint4*>(dst + k * 8) = w;
                     }
                 }
@@ -419,7 +436,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // Two halves of 32 query rows, each its own bulk group: the rows of one half are rewritten
             // while the bulk engine is still reading the other half of the previous step.
             const int nq = min(64, L - q0);
-            float* dst = p.dq_acc + (static_cast<size_t>(h) * p.T + r0 + q0) * D;
+            float* dst = p.dq_acc + (static_cast<size_t>(h) * p.T + sp.gt0 + q0) * D;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 if (x == 0) bulk_wait_read<1>();  // the group that last read this half has finished reading
@@ -454,8 +471,8 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             mbar_arrive_expect_tx(kv_full, 2 * Cfg::kTileBytes);
 #pragma unroll
             for (int a = 0; a < D / 64; ++a) {
-                tma_load_3d(sK + a * Cfg::kAtomBytes, &map_k, kv_full, a * 64, g, r0 + kv0);
-                tma_load_3d(sV + a * Cfg::kAtomBytes, &map_v, kv_full, a * 64, g, r0 + kv0);
+                SDPA_TMA_LOAD_ROWS(sK + a * Cfg::kAtomBytes, &map_k, kv_full, a * 64, r0 + kv0, g, sp.bidx, p.lay.dense);
+                SDPA_TMA_LOAD_ROWS(sV + a * Cfg::kAtomBytes, &map_v, kv_full, a * 64, r0 + kv0, g, sp.bidx, p.lay.dense);
             }
         }
         bool ok = true;
@@ -471,9 +488,9 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 mbar_arrive_expect_tx(&q_full[st], Cfg::kStageBytes);
 #pragma unroll
                 for (int a = 0; a < D / 64; ++a) {
-                    tma_load_3d(dst + a * Cfg::kStepAtomBytes, &map_q, &q_full[st], a * 64, h, r0 + q0);
-                    tma_load_3d(dst + Cfg::kStepBytes + a * Cfg::kStepAtomBytes, &map_do, &q_full[st], a * 64, h,
-                                r0 + q0);
+                    SDPA_TMA_LOAD_ROWS(dst + a * Cfg::kStepAtomBytes, &map_q, &q_full[st], a * 64, r0 + q0, h, sp.bidx, p.lay.dense);
+                    SDPA_TMA_LOAD_ROWS(dst + Cfg::kStepBytes + a * Cfg::kStepAtomBytes, &map_do, &q_full[st], a * 64, r0 + q0,
+                                h, sp.bidx, p.lay.dense);
                 }
             }
             float* rows = sRows + st * 128;
@@ -482,9 +499,9 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const int qi = lane * 2 + e;
                 float lv = INFINITY, dv = 0.f;  // rows past the sequence end: P = exp2(-inf) = 0
                 if (q0 + qi < L) {
-                    const size_t idx = static_cast<size_t>(h) * p.T + r0 + q0 + qi;
-                    lv = p.lse[idx] * 1.4426950408889634f;
-                    dv = p.delta[idx];
+                    lv = p.lse[sp.bidx * p.lay.lse_bs + static_cast<long long>(h) * p.lay.lse_hs + r0 + q0 + qi] *
+                         1.4426950408889634f;
+                    dv = p.delta[static_cast<size_t>(h) * p.T + sp.gt0 + q0 + qi];
                 }
                 rows[qi] = lv;
                 rows[64 + qi] = dv;

@@ -16,6 +16,7 @@
 // the stale max stays the reference, which changes nothing in exact arithmetic.
 #pragma once
 #include "ptx.cuh"
+#include "layout.cuh"
 
 #ifndef SDPA_TR
 #define SDPA_TR(role, it, k) do { } while (0)
@@ -38,6 +39,7 @@ struct FwdParams {
     int causal;
     int max_seqlen;
     int d;             // head dimension of the tensors (multiple of 8, <= D of the kernel; columns d..D-1 are zero padding)
+    TensorLayout lay;  // strides of q / o (and of k / v for the non-paged kernel), lse
     int head_chunk;    // (sequence, query head) pairs whose CTAs are launched interleaved
     float scale;       // softmax scale
     float scale_log2;  // scale * log2(e)
@@ -98,13 +100,13 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int b = bh / p.Hq, h = bh % p.Hq;
     const int g = h / (p.Hq / p.Hkv);
     const int pair = n_pairs_grid - 1 - pair_raw;  // heaviest (latest) query tiles first
-    const int r0 = p.cu_seqlens[b];
-    const int r1 = p.cu_seqlens[b + 1];
-    int L = r1 - r0;
-    if (L < 0 || r0 < 0 || r1 > p.T || L > p.max_seqlen) {
+    SeqPos sp;
+    if (!locate_sequence(p.lay, p.cu_seqlens, b, p.T, p.max_seqlen, sp)) {
         if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
         return;
     }
+    const int r0 = sp.tok0;  // token coordinate of the sequence's first row
+    const int L = sp.L;
     const int q_start = pair * 256;
     if (q_start >= L) return;
     int Lk = L, kbase = 0;  // number of keys of this sequence; first entry of its page list
@@ -328,12 +330,15 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const int rr = (warp & 3) * 32 + pass * kRowsPerPass + lane / kChunks;  // row inside the tile
                     if (rr < rows_left && k * 8 < p.d) {
                         const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * (D * 2) + ((k ^ (rr & 7)) << 4));
-                        __nv_bfloat16* dst = p.o + (static_cast<size_t>(r0 + q_start + t * 128 + rr) * p.Hq + h) * p.d;
+                        __nv_bfloat16* dst = p.o + sp.bidx * p.lay.bs_q +
+                                             static_cast<long long>(r0 + q_start + t * 128 + rr) * p.lay.ts_q +
+                                             static_cast<long long>(h) * p.lay.hs_q;
                         *reinterpret_cast<uint4*>(dst + k * 8) = w;
                     }
                 }
             }
-            if (valid) p.lse[static_cast<size_t>(h) * p.T + r0 + row] = m * p.scale + logf(l);
+            if (valid)
+                p.lse[sp.bidx * p.lay.lse_bs + static_cast<long long>(h) * p.lay.lse_hs + r0 + row] = m * p.scale + logf(l);
         }
     } else {
         setmaxnreg_dec<80>();
@@ -346,13 +351,14 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (lane == 0) {
                 mbar_arrive_expect_tx(&q_full[0], Cfg::kTileBytes);
 #pragma unroll
-                for (int a = 0; a < D / 64; ++a) tma_load_3d(sQ + a * Cfg::kAtomBytes, &map_q, &q_full[0], a * 64, h, r0 + q_start);
+                for (int a = 0; a < D / 64; ++a)
+                    SDPA_TMA_LOAD_ROWS(sQ + a * Cfg::kAtomBytes, &map_q, &q_full[0], a * 64, r0 + q_start, h, sp.bidx, p.lay.dense);
                 if (n_kv[1] > 0) {
                     mbar_arrive_expect_tx(&q_full[1], Cfg::kTileBytes);
 #pragma unroll
                     for (int a = 0; a < D / 64; ++a)
-                        tma_load_3d(sQ + Cfg::kTileBytes + a * Cfg::kAtomBytes, &map_q, &q_full[1], a * 64, h,
-                                    r0 + q_start + 128);
+                        SDPA_TMA_LOAD_ROWS(sQ + Cfg::kTileBytes + a * Cfg::kAtomBytes, &map_q, &q_full[1], a * 64,
+                                    r0 + q_start + 128, h, sp.bidx, p.lay.dense);
                 }
             }
             bool ok = true;
@@ -412,7 +418,8 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 auto load_tile = [&](const CUtensorMap* map, uint8_t* dst, uint64_t* bar, int head, int tok) {
                     mbar_arrive_expect_tx(bar, Cfg::kTileBytes);
 #pragma unroll
-                    for (int a = 0; a < D / 64; ++a) tma_load_3d(dst + a * Cfg::kAtomBytes, map, bar, a * 64, head, tok);
+                    for (int a = 0; a < D / 64; ++a)
+                        SDPA_TMA_LOAD_ROWS(dst + a * Cfg::kAtomBytes, map, bar, a * 64, tok, head, sp.bidx, p.lay.dense);
                 };
                 bool ok = true;
                 load_tile(&map_q, sQ, &q_full[0], h, r0 + q_start);
@@ -421,9 +428,6 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const int st = it % S;
                         ok = mbar_wait(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
                         if (!ok) break;
-#ifdef SDPA_EXP_NO_KV_RELOAD
-                        if (it >= S) mbar_arrive(&kv_full[st]); else
-#endif
                         load_tile(kv == 0 ? &map_k : &map_v, sRing + st * Cfg::kTileBytes, &kv_full[st], g,
                                   r0 + j * 128);
                         if (j == 0 && kv == 0 && n_kv[1] > 0)

@@ -93,13 +93,25 @@ static int device_state(DeviceState** out) {
     return st.arch_ok ? SDPA_OK : SDPA_ERR_ARCH;
 }
 
-// Tensor map over a packed bf16 [T, H, D] tensor: dims {D, H, T}, box {64, 1, rows}, 128B swizzle.
-static int make_map(CUtensorMap* map, const void* base, int T, int H, int D, int box_rows) {
-    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(T)};
-    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(H) * D * 2};
-    const cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+// Tensor map over a bf16 attention tensor with H heads, box = box_rows rows of 64 columns, 128B swizzle.
+// Packed [T, H, D]: dims {D, H, T, 1}, box {64, 1, rows, 1}.  Dense [B, H, S, D]: dims {D, S, H, B}, box
+// {64, rows, 1, 1}.  Both keep the strides increasing and give the same [rows][64] tile in shared memory.
+static int make_map(CUtensorMap* map, const void* base, const TensorLayout& lay, int n_batch, int rows, int H, int D,
+                    int box_rows) {
+    cuuint64_t dims[4], strides[3];
+    cuuint32_t box[4];
+    const cuuint64_t u = static_cast<cuuint64_t>(D) * 2;
+    if (lay.dense) {
+        dims[0] = D; dims[1] = rows; dims[2] = H; dims[3] = n_batch;
+        strides[0] = u; strides[1] = u * rows; strides[2] = u * rows * H;
+        box[0] = 64; box[1] = box_rows; box[2] = 1; box[3] = 1;
+    } else {
+        dims[0] = D; dims[1] = H; dims[2] = rows; dims[3] = 1;
+        strides[0] = u; strides[1] = u * H; strides[2] = u * H * rows;
+        box[0] = 64; box[1] = 1; box[2] = box_rows; box[3] = 1;
+    }
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -109,14 +121,31 @@ static int make_map(CUtensorMap* map, const void* base, int T, int H, int D, int
     return SDPA_OK;
 }
 
+static TensorLayout packed_layout(int T, int Hq, int Hkv, int D) {
+    TensorLayout l{};
+    l.ts_q = Hq * D; l.hs_q = D; l.ts_kv = Hkv * D; l.hs_kv = D;
+    l.lse_hs = T; l.lse_bs = 0; l.bs_q = 0; l.bs_kv = 0;
+    l.dense = 0; l.S = T > 0 ? T : 1; l.has_lengths = 1;
+    return l;
+}
+static TensorLayout dense_layout(int Hq, int Hkv, int S, int D, bool has_lengths) {
+    TensorLayout l{};
+    l.ts_q = D; l.hs_q = S * D; l.ts_kv = D; l.hs_kv = S * D;
+    l.bs_q = static_cast<long long>(Hq) * S * D; l.bs_kv = static_cast<long long>(Hkv) * S * D;
+    l.lse_hs = S; l.lse_bs = static_cast<long long>(Hq) * S;
+    l.dense = 1; l.S = S; l.has_lengths = has_lengths ? 1 : 0;
+    return l;
+}
+
 // Head dimension the kernels are instantiated for: 64 or 128; a smaller head dimension runs in the next
 // larger kernel, its missing columns zero-filled by the TMA loads (out-of-bounds box columns read as 0).
 static int padded_head_dim(int D) { return D <= 64 ? 64 : 128; }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-static int check_common(const int32_t* cu, int B, int Hq, int Hkv, int D, float scale, int T, int max_seqlen) {
-    if (cu == nullptr) return SDPA_ERR_NULL;
+static int check_common(const int32_t* cu, int B, int Hq, int Hkv, int D, float scale, int T, int max_seqlen,
+                        bool cu_optional = false) {
+    if (cu == nullptr && !cu_optional) return SDPA_ERR_NULL;
     if (B < 1 || Hq < 1 || Hkv < 1 || T < 0 || max_seqlen < 0) return SDPA_ERR_SHAPE;
     if (D < 8 || D > 128 || (D % 8) != 0) return SDPA_ERR_SHAPE;
     if (Hq % Hkv != 0) return SDPA_ERR_SHAPE;
@@ -160,10 +189,10 @@ static size_t bwd_delta_bytes(int Hq, int T) { return align_up(static_cast<size_
 
 using namespace sdpa;
 
-extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, float* lse, const int32_t* cu_seqlens,
-                        int B, int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
-                        void* stream) {
-    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen);
+static int fwd_launch(const void* q, const void* k, const void* v, void* o, float* lse, const int32_t* cu_seqlens,
+                      int B, int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
+                      void* stream, const TensorLayout& lay) {
+    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen, lay.dense != 0);
     if (rc != SDPA_OK) return rc;
     if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
     if (!q || !k || !v || !o || !lse) return SDPA_ERR_NULL;
@@ -174,11 +203,13 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
     if (rc != SDPA_OK) return rc;
 
     CUtensorMap mq, mk, mv;
-    if ((rc = make_map(&mq, q, total_tokens, Hq, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mk, k, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mv, v, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
+    const int map_rows = lay.dense ? lay.S : total_tokens;
+    if ((rc = make_map(&mq, q, lay, B, map_rows, Hq, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mk, k, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mv, v, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
 
     FwdParams p;
+    p.lay = lay;
     p.cu_seqlens = cu_seqlens;
     p.kv_indptr = nullptr; p.kv_indices = nullptr; p.k_cache = nullptr; p.v_cache = nullptr; p.num_pages = 0;
     p.o = static_cast<__nv_bfloat16*>(o);
@@ -205,6 +236,29 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
     return SDPA_OK;
 }
 
+extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, float* lse, const int32_t* cu_seqlens,
+                        int B, int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
+                        void* stream) {
+    return fwd_launch(q, k, v, o, lse, cu_seqlens, B, Hq, Hkv, D, causal, scale, total_tokens, max_seqlen, stream,
+                      packed_layout(total_tokens, Hq, Hkv, D));
+}
+
+// Limits of the dense entry points: B * S rows are indexed with 32-bit integers.
+static int check_dense(int B, int S) {
+    if (B < 1 || S < 0) return SDPA_ERR_SHAPE;
+    if (static_cast<long long>(B) * S > 2147483647ll) return SDPA_ERR_SHAPE;
+    return SDPA_OK;
+}
+
+extern "C" int sdpa_fwd_bhsd(const void* q, const void* k, const void* v, void* o, float* lse,
+                             const int32_t* cu_seqlens, int B, int Hq, int Hkv, int S, int D, int causal, float scale,
+                             void* stream) {
+    const int rc = check_dense(B, S);
+    if (rc != SDPA_OK) return rc;
+    return fwd_launch(q, k, v, o, lse, cu_seqlens, B, Hq, Hkv, D, causal, scale, B * S, S, stream,
+                      dense_layout(Hq, Hkv, S, D, cu_seqlens != nullptr));
+}
+
 extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
                               const int32_t* cu_seqlens_q, const int32_t* kv_indptr, const int32_t* kv_indices, int B,
                               int Hq, int Hkv, int D, int causal, float scale, int total_q, int max_seqlen_q,
@@ -222,8 +276,10 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
     rc = device_state(&st);
     if (rc != SDPA_OK) return rc;
     CUtensorMap mq;
-    if ((rc = make_map(&mq, q, total_q, Hq, D, 128)) != SDPA_OK) return rc;
+    const TensorLayout lay = packed_layout(total_q, Hq, Hkv, D);
+    if ((rc = make_map(&mq, q, lay, 1, total_q, Hq, D, 128)) != SDPA_OK) return rc;
     FwdParams p;
+    p.lay = lay;
     p.cu_seqlens = cu_seqlens_q;
     p.kv_indptr = kv_indptr;
     p.kv_indices = kv_indices;
@@ -261,11 +317,11 @@ extern "C" size_t sdpa_bwd_workspace_bytes(int B, int Hq, int Hkv, int D, int to
     return bwd_dq_bytes(Hq, padded_head_dim(D), total_tokens) + bwd_delta_bytes(Hq, total_tokens) + 256;
 }
 
-extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
-                        void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D,
-                        int causal, float scale, int total_tokens, int max_seqlen, void* workspace,
-                        size_t workspace_bytes, void* stream) {
-    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen);
+static int bwd_launch(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
+                      void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D,
+                      int causal, float scale, int total_tokens, int max_seqlen, void* workspace,
+                      size_t workspace_bytes, void* stream, const TensorLayout& lay) {
+    int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen, lay.dense != 0);
     if (rc != SDPA_OK) return rc;
     if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
     if (!q || !k || !v || !o || !lse || !dout || !dq || !dk || !dv) return SDPA_ERR_NULL;
@@ -293,21 +349,23 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
         if (Dp == 128)
             sdpa_bwd_preprocess_kernel<128><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
                 static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
-                total_tokens, Hq, D);
+                total_tokens, Hq, D, lay);
         else
             sdpa_bwd_preprocess_kernel<64><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
                 static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
-                total_tokens, Hq, D);
+                total_tokens, Hq, D, lay);
         SDPA_CUDA_TRY(cudaGetLastError());
     }
 
     CUtensorMap mq, mk, mv, mdo;
-    if ((rc = make_map(&mq, q, total_tokens, Hq, D, 64)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mk, k, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mv, v, total_tokens, Hkv, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mdo, dout, total_tokens, Hq, D, 64)) != SDPA_OK) return rc;
+    const int map_rows = lay.dense ? lay.S : total_tokens;
+    if ((rc = make_map(&mq, q, lay, B, map_rows, Hq, D, 64)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mk, k, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mv, v, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mdo, dout, lay, B, map_rows, Hq, D, 64)) != SDPA_OK) return rc;
 
     BwdParams p;
+    p.lay = lay;
     p.cu_seqlens = cu_seqlens;
     p.lse = lse;
     p.delta = delta;
@@ -343,10 +401,28 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
         const int threads = 256;
         const long long blocks = (n8 + threads - 1) / threads;
         sdpa_bwd_dq_convert_kernel<<<static_cast<unsigned>(blocks), threads, 0, s>>>(
-            dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale, total_tokens, Hq, Dp, D);
+            dq_acc, static_cast<__nv_bfloat16*>(dq), n8, scale, total_tokens, Hq, Dp, D, lay);
         SDPA_CUDA_TRY(cudaGetLastError());
     }
     return SDPA_OK;
+}
+
+extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
+                        void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D,
+                        int causal, float scale, int total_tokens, int max_seqlen, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    return bwd_launch(q, k, v, o, lse, dout, dq, dk, dv, cu_seqlens, B, Hq, Hkv, D, causal, scale, total_tokens,
+                      max_seqlen, workspace, workspace_bytes, stream, packed_layout(total_tokens, Hq, Hkv, D));
+}
+
+extern "C" int sdpa_bwd_bhsd(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                             const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq,
+                             int Hkv, int S, int D, int causal, float scale, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+    const int rc = check_dense(B, S);
+    if (rc != SDPA_OK) return rc;
+    return bwd_launch(q, k, v, o, lse, dout, dq, dk, dv, cu_seqlens, B, Hq, Hkv, D, causal, scale, B * S, S,
+                      workspace, workspace_bytes, stream, dense_layout(Hq, Hkv, S, D, cu_seqlens != nullptr));
 }
 
 // ------------------------------------------------------------------ built-in scratch (no allocation)
