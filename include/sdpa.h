@@ -177,12 +177,17 @@ int sdpa_bwd_static_scratch(const void* q, const void* k, const void* v, const v
 /*
  * Whole step with HOST buffers (no counterpart in the paper's operator list beyond composing the
  * forward and backward workloads of its appendix "Workloads"): copies q, k, v, dout and cu_seqlens
- * from host memory to the device, runs sdpa_fwd then sdpa_bwd, and copies o, lse, dq, dk, dv back,
- * all asynchronously on `stream`.  Host pointers should be page-locked for the copies to overlap;
- * layouts are those of sdpa_fwd / sdpa_bwd.  `staging` is caller-owned, 256-byte aligned DEVICE
- * scratch of at least sdpa_host_staging_bytes(...) bytes that holds the device copies and the
- * backward workspace; the library allocates nothing.  The host outputs are valid once the stream
- * has been synchronised.
+ * from host memory to the device, runs sdpa_fwd then sdpa_bwd, and copies o, lse, dq, dk, dv back.
+ * The work is ordered like any other work on `stream`: it starts after what was enqueued on `stream`
+ * before the call, and what is enqueued on `stream` after the call starts when the host outputs are
+ * complete; the host outputs are valid once the stream has been synchronised.  Inside, the step is cut
+ * into up to four chunks of kv heads that are copied in, computed and copied out in a pipeline (compute
+ * on `stream`, the copies on two internal non-blocking streams that fork from and join `stream` through
+ * events), so that the two directions of the host link work at the same time.  The internal streams and
+ * events are created on the calling thread's first call on a device (no device memory is allocated) and
+ * kept.  Host pointers should be page-locked for the copies to overlap; layouts are those of sdpa_fwd /
+ * sdpa_bwd.  `staging` is caller-owned, 256-byte aligned DEVICE scratch of at least
+ * sdpa_host_staging_bytes(...) bytes that holds the device copies and the backward workspace.
  */
 size_t sdpa_host_staging_bytes(int B, int Hq, int Hkv, int D, int total_tokens, int max_seqlen);
 int sdpa_fwd_bwd_host(const void* q, const void* k, const void* v, const void* dout, void* o,

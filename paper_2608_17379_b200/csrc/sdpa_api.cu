@@ -479,11 +479,48 @@ extern "C" size_t sdpa_host_staging_bytes(int B, int Hq, int Hkv, int D, int tot
     const size_t ws = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
     if (ws == 0) return 0;
     const size_t T = static_cast<size_t>(total_tokens);
-    const size_t qb = align_up(T * Hq * D * 2, 256), kb = align_up(T * Hkv * D * 2, 256);
-    const size_t lb = align_up(T * Hq * 4, 256), cb = align_up(static_cast<size_t>(B + 1) * 4, 256);
-    return 4 * qb /* q, o, dout, dq */ + 4 * kb /* k, v, dk, dv */ + lb + cb + ws;
+    const size_t qb = T * Hq * D * 2, kb = T * Hkv * D * 2, lb = T * Hq * 4;
+    const size_t cb = align_up(static_cast<size_t>(B + 1) * 4, 256);
+    // q, dout, o, dq + k, v, dk, dv + lse, cut into at most 8 chunks of 9 separately aligned pieces
+    return 4 * qb + 4 * kb + lb + cb + align_up(ws, 256) + 8 * 9 * 256;
 }
 
+// Copy streams and events of sdpa_fwd_bwd_host, one set per (host thread, device), created on first use
+// and kept for the life of the thread.
+constexpr int kHostMaxChunks = 8;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr;
+    cudaEvent_t ev_in[kHostMaxChunks] = {}, ev_cmp[kHostMaxChunks] = {};
+};
+static thread_local HostPipe tl_pipe[sdpa::kMaxDevices];
+
+static int host_pipe(HostPipe** out) {
+    int dev = -1;
+    SDPA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= sdpa::kMaxDevices) return SDPA_ERR_ARCH;
+    HostPipe& hp = tl_pipe[dev];
+    if (!hp.ready) {
+        SDPA_CUDA_TRY(cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking));
+        SDPA_CUDA_TRY(cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking));
+        SDPA_CUDA_TRY(cudaEventCreateWithFlags(&hp.ev_start, cudaEventDisableTiming));
+        SDPA_CUDA_TRY(cudaEventCreateWithFlags(&hp.ev_out, cudaEventDisableTiming));
+        for (int i = 0; i < kHostMaxChunks; ++i) {
+            SDPA_CUDA_TRY(cudaEventCreateWithFlags(&hp.ev_in[i], cudaEventDisableTiming));
+            SDPA_CUDA_TRY(cudaEventCreateWithFlags(&hp.ev_cmp[i], cudaEventDisableTiming));
+        }
+        hp.ready = true;
+    }
+    *out = &hp;
+    return SDPA_OK;
+}
+
+// The step is cut into chunks of kv heads (with their query heads): heads are independent problems, so
+// while chunk c computes on the caller's stream, chunk c+1 is copied in on one copy stream and chunk c-1
+// is copied out on another.  PCIe is full duplex, so the step costs about max(copy in, copy out) instead
+// of their sum.  Chunks are taken out of the host tensors with pitched copies ([T, H, D] rows, a head
+// range per chunk) and live on the device as contiguous [T, Hc, D] tensors.
 extern "C" int sdpa_fwd_bwd_host(const void* q, const void* k, const void* v, const void* dout, void* o, float* lse,
                                  void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv,
                                  int D, int causal, float scale, int total_tokens, int max_seqlen, void* staging,
@@ -495,34 +532,70 @@ extern "C" int sdpa_fwd_bwd_host(const void* q, const void* k, const void* v, co
     const size_t need = sdpa_host_staging_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
     if (staging == nullptr || (reinterpret_cast<uintptr_t>(staging) & 255u) || staging_bytes < need)
         return SDPA_ERR_WORKSPACE;
+    HostPipe* hp = nullptr;
+    if ((rc = host_pipe(&hp)) != SDPA_OK) return rc;
+
     const size_t T = static_cast<size_t>(total_tokens);
-    const size_t q_bytes = T * Hq * D * 2, k_bytes = T * Hkv * D * 2, l_bytes = T * Hq * 4;
+    const int G = Hq / Hkv;
+    const int n_chunks = Hkv < 4 ? Hkv : 4;
+    const size_t row = static_cast<size_t>(D) * 2;  // bytes of one head row
     const size_t c_bytes = static_cast<size_t>(B + 1) * 4;
-    const size_t qb = align_up(q_bytes, 256), kb = align_up(k_bytes, 256);
-    const size_t lb = align_up(l_bytes, 256), cb = align_up(c_bytes, 256);
     uint8_t* base = static_cast<uint8_t*>(staging);
-    uint8_t* d_q = base;            uint8_t* d_o = d_q + qb;   uint8_t* d_do = d_o + qb;  uint8_t* d_dq = d_do + qb;
-    uint8_t* d_k = d_dq + qb;       uint8_t* d_v = d_k + kb;   uint8_t* d_dk = d_v + kb;  uint8_t* d_dv = d_dk + kb;
-    uint8_t* d_lse = d_dv + kb;     uint8_t* d_cu = d_lse + lb; uint8_t* d_ws = d_cu + cb;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { uint8_t* p = base + off; off += align_up(bytes, 256); return p; };
+    uint8_t* d_cu = take(c_bytes);
+    // the backward workspace is shared by the chunks (they run one after the other on the caller's stream)
     const size_t ws_bytes = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen);
+    uint8_t* d_ws = take(ws_bytes);
+
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    SDPA_CUDA_TRY(cudaMemcpyAsync(d_cu, cu_seqlens, c_bytes, cudaMemcpyHostToDevice, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(d_q, q, q_bytes, cudaMemcpyHostToDevice, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(d_k, k, k_bytes, cudaMemcpyHostToDevice, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(d_v, v, k_bytes, cudaMemcpyHostToDevice, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(d_do, dout, q_bytes, cudaMemcpyHostToDevice, s));
-    rc = sdpa_fwd(d_q, d_k, d_v, d_o, reinterpret_cast<float*>(d_lse), reinterpret_cast<const int32_t*>(d_cu), B, Hq,
-                  Hkv, D, causal, scale, total_tokens, max_seqlen, stream);
-    if (rc != SDPA_OK) return rc;
-    rc = sdpa_bwd(d_q, d_k, d_v, d_o, reinterpret_cast<const float*>(d_lse), d_do, d_dq, d_dk, d_dv,
-                  reinterpret_cast<const int32_t*>(d_cu), B, Hq, Hkv, D, causal, scale, total_tokens, max_seqlen, d_ws,
-                  ws_bytes, stream);
-    if (rc != SDPA_OK) return rc;
-    SDPA_CUDA_TRY(cudaMemcpyAsync(o, d_o, q_bytes, cudaMemcpyDeviceToHost, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(lse, d_lse, l_bytes, cudaMemcpyDeviceToHost, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(dq, d_dq, q_bytes, cudaMemcpyDeviceToHost, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(dk, d_dk, k_bytes, cudaMemcpyDeviceToHost, s));
-    SDPA_CUDA_TRY(cudaMemcpyAsync(dv, d_dv, k_bytes, cudaMemcpyDeviceToHost, s));
+    SDPA_CUDA_TRY(cudaEventRecord(hp->ev_start, s));
+    SDPA_CUDA_TRY(cudaStreamWaitEvent(hp->s_in, hp->ev_start, 0));
+    SDPA_CUDA_TRY(cudaMemcpyAsync(d_cu, cu_seqlens, c_bytes, cudaMemcpyHostToDevice, hp->s_in));
+    for (int c = 0; c < n_chunks; ++c) {
+        const int g0 = static_cast<int>(static_cast<long long>(Hkv) * c / n_chunks);
+        const int g1 = static_cast<int>(static_cast<long long>(Hkv) * (c + 1) / n_chunks);
+        const int hk = g1 - g0, hq = hk * G, h0 = g0 * G;
+        const size_t qw = hq * row, kw = hk * row;  // bytes per token of the chunk's q-like / k-like tensors
+        uint8_t* d_q = take(T * qw); uint8_t* d_do = take(T * qw); uint8_t* d_o = take(T * qw); uint8_t* d_dq = take(T * qw);
+        uint8_t* d_k = take(T * kw); uint8_t* d_v = take(T * kw); uint8_t* d_dk = take(T * kw); uint8_t* d_dv = take(T * kw);
+        uint8_t* d_lse = take(T * hq * 4);
+        if (off > staging_bytes) return SDPA_ERR_WORKSPACE;
+        const size_t qp = static_cast<size_t>(Hq) * row, kp = static_cast<size_t>(Hkv) * row;  // host pitches
+        const uint8_t* hq_src = static_cast<const uint8_t*>(q) + h0 * row;
+        const uint8_t* hdo_src = static_cast<const uint8_t*>(dout) + h0 * row;
+        const uint8_t* hk_src = static_cast<const uint8_t*>(k) + g0 * row;
+        const uint8_t* hv_src = static_cast<const uint8_t*>(v) + g0 * row;
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(d_q, qw, hq_src, qp, qw, T, cudaMemcpyHostToDevice, hp->s_in));
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(d_k, kw, hk_src, kp, kw, T, cudaMemcpyHostToDevice, hp->s_in));
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(d_v, kw, hv_src, kp, kw, T, cudaMemcpyHostToDevice, hp->s_in));
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(d_do, qw, hdo_src, qp, qw, T, cudaMemcpyHostToDevice, hp->s_in));
+        SDPA_CUDA_TRY(cudaEventRecord(hp->ev_in[c], hp->s_in));
+
+        SDPA_CUDA_TRY(cudaStreamWaitEvent(s, hp->ev_in[c], 0));
+        rc = sdpa_fwd(d_q, d_k, d_v, d_o, reinterpret_cast<float*>(d_lse), reinterpret_cast<const int32_t*>(d_cu), B, hq,
+                      hk, D, causal, scale, total_tokens, max_seqlen, stream);
+        if (rc != SDPA_OK) return rc;
+        rc = sdpa_bwd(d_q, d_k, d_v, d_o, reinterpret_cast<const float*>(d_lse), d_do, d_dq, d_dk, d_dv,
+                      reinterpret_cast<const int32_t*>(d_cu), B, hq, hk, D, causal, scale, total_tokens, max_seqlen,
+                      d_ws, ws_bytes, stream);
+        if (rc != SDPA_OK) return rc;
+        SDPA_CUDA_TRY(cudaEventRecord(hp->ev_cmp[c], s));
+
+        SDPA_CUDA_TRY(cudaStreamWaitEvent(hp->s_out, hp->ev_cmp[c], 0));
+        uint8_t* ho = static_cast<uint8_t*>(o) + h0 * row;
+        uint8_t* hdq = static_cast<uint8_t*>(dq) + h0 * row;
+        uint8_t* hdk = static_cast<uint8_t*>(dk) + g0 * row;
+        uint8_t* hdv = static_cast<uint8_t*>(dv) + g0 * row;
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(ho, qp, d_o, qw, qw, T, cudaMemcpyDeviceToHost, hp->s_out));
+        SDPA_CUDA_TRY(cudaMemcpyAsync(lse + static_cast<size_t>(h0) * T, d_lse, T * hq * 4, cudaMemcpyDeviceToHost, hp->s_out));
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(hdq, qp, d_dq, qw, qw, T, cudaMemcpyDeviceToHost, hp->s_out));
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(hdk, kp, d_dk, kw, kw, T, cudaMemcpyDeviceToHost, hp->s_out));
+        SDPA_CUDA_TRY(cudaMemcpy2DAsync(hdv, kp, d_dv, kw, kw, T, cudaMemcpyDeviceToHost, hp->s_out));
+    }
+    // join: everything after this call on the caller's stream sees the finished host outputs
+    SDPA_CUDA_TRY(cudaEventRecord(hp->ev_out, hp->s_out));
+    SDPA_CUDA_TRY(cudaStreamWaitEvent(s, hp->ev_out, 0));
     return SDPA_OK;
 }
 

@@ -244,8 +244,13 @@ def test_a_wait_that_runs_out_reports_timeout_and_the_context_survives():
     run_and_compare(TL.random_workload((200,), 2, 2, 64, True, seed=61))  # the library still works
 
 
-def test_host_buffer_entry_point_matches_device_entry_points():
-    w = TL.random_workload((333, 200), 4, 2, 128, True, seed=60)
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 128), (12, 6, 64), (3, 1, 128), (10, 5, 96), (16, 8, 128)])
+def test_host_buffer_entry_point_matches_device_entry_points(Hq, Hkv, D):
+    """The host entry point cuts the step into chunks of kv heads and pipelines copies and compute; heads
+    are independent, so the result must equal the one-shot device result (several chunkings covered:
+    fewer kv heads than chunks, uneven chunks, two heads per chunk).  Called twice in a row on one
+    stream: the second call reuses the staging buffer."""
+    w = TL.random_workload((333, 200), Hq, Hkv, D, True, seed=60)
     qb, kb, vb, dob = W.make_inputs(w)
     ref = TL.run_gpu(qb, kb, vb, dob, w.cu_seqlens, w.max_seqlen, True, w.scale)
     host = [torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in (qb, kb, vb, dob)]
@@ -256,8 +261,10 @@ def test_host_buffer_entry_point_matches_device_entry_points():
     dk = torch.empty((T, Hkv, D), dtype=torch.bfloat16).pin_memory(); dv = torch.empty_like(dk).pin_memory()
     staging = torch.empty(binding.sdpa_host_staging_bytes(w.B, Hq, Hkv, D, T, w.max_seqlen), dtype=torch.uint8,
                           device="cuda")
-    binding.sdpa_fwd_bwd_host(host[0], host[1], host[2], host[3], o, lse, dq, dk, dv, torch.from_numpy(w.cu_seqlens),
-                              w.max_seqlen, True, w.scale, staging)
+    for _ in range(2):
+        binding.sdpa_fwd_bwd_host(host[0], host[1], host[2], host[3], o, lse, dq, dk, dv,
+                                  torch.from_numpy(w.cu_seqlens), w.max_seqlen, True, w.scale, staging)
+    torch.cuda.synchronize()
     assert binding.query_status() == (0, 0)
     assert torch.equal(o.view(torch.int16), ref["o"].cpu().view(torch.int16))
     assert torch.equal(lse, ref["lse"].cpu())
