@@ -117,6 +117,23 @@ int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * sdpa_bwd with a reproducible dq (the paper's backward workloads do not ask for this; the libraries it
+ * compares with offer such a mode).  sdpa_bwd adds the dq contributions of the key tiles of a sequence
+ * with fp32 reduce-adds in whatever order the tiles get there, so the last bits of dq can differ from run
+ * to run (dk and dv never do).  This entry point makes the key tiles take turns on every 64-row block of
+ * queries, from the highest key tile down, through per-block turn counters in the workspace: two calls on
+ * the same inputs give bit-identical dq, dk, dv (dk and dv equal those of sdpa_bwd bit for bit).  Same
+ * arguments, workspace size, errors and status reporting as sdpa_bwd.  It is slower because the key tiles
+ * with the fewest visible queries have to be launched first instead of last (the tiles waited for must be
+ * running already), which balances the SMs less well.  A turn wait is bounded like every other
+ * device-side wait (SDPA_STATUS_TIMEOUT).
+ */
+int sdpa_bwd_deterministic(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                           const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens,
+                           int B, int Hq, int Hkv, int D, int causal, float scale, int total_tokens,
+                           int max_seqlen, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The same forward and backward passes on dense tensors in the shape convention of the paper's attention
  * workloads (appendix "Workloads": bf16 tensors of shape [batch, heads, sequence, head dim]):
  *        q, o, dout, dq : bf16 [B, Hq,  S, D]      k, v, dk, dv : bf16 [B, Hkv, S, D]

@@ -19,7 +19,7 @@ SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
            "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout", "sdpa_fwd_paged",
-           "sdpa_fwd_bhsd", "sdpa_bwd_bhsd")
+           "sdpa_fwd_bhsd", "sdpa_bwd_bhsd", "sdpa_bwd_deterministic")
 
 
 class SdpaError(RuntimeError):
@@ -42,6 +42,8 @@ def load():
     lib.sdpa_bwd_workspace_bytes.argtypes = [ci] * 6
     lib.sdpa_bwd.restype = ci
     lib.sdpa_bwd.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp, ctypes.c_size_t, vp]
+    lib.sdpa_bwd_deterministic.restype = ci
+    lib.sdpa_bwd_deterministic.argtypes = lib.sdpa_bwd.argtypes
     lib.sdpa_host_staging_bytes.restype = ctypes.c_size_t
     lib.sdpa_host_staging_bytes.argtypes = [ci] * 6
     lib.sdpa_fwd_bwd_host.restype = ci
@@ -120,8 +122,9 @@ def sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_tokens, max_seqlen) -> int:
 
 
 def sdpa_bwd(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, scale: float,
-             dq=None, dk=None, dv=None, workspace=None, stream=None):
-    """Gradients (dq, dk, dv) bf16 of sum(dout * O); o and lse are the outputs of sdpa_fwd."""
+             dq=None, dk=None, dv=None, workspace=None, stream=None, deterministic: bool = False):
+    """Gradients (dq, dk, dv) bf16 of sum(dout * O); o and lse are the outputs of sdpa_fwd.
+    deterministic=True calls sdpa_bwd_deterministic (bit-reproducible dq)."""
     lib = load()
     T, Hq, Hkv, D = _dims(q, k)
     B = cu_seqlens.numel() - 1
@@ -134,10 +137,11 @@ def sdpa_bwd(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, s
         dk = torch.empty_like(k)
     if dv is None:
         dv = torch.empty_like(v)
-    rc = lib.sdpa_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
-                      _ptr(cu_seqlens), B, Hq, Hkv, D, int(bool(causal)), float(scale), T, int(max_seqlen),
-                      _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
-    _check(rc, "sdpa_bwd")
+    fn = lib.sdpa_bwd_deterministic if deterministic else lib.sdpa_bwd
+    rc = fn(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
+            _ptr(cu_seqlens), B, Hq, Hkv, D, int(bool(causal)), float(scale), T, int(max_seqlen),
+            _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
+    _check(rc, "sdpa_bwd_deterministic" if deterministic else "sdpa_bwd")
     return dq, dk, dv
 
 

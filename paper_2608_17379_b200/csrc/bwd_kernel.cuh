@@ -43,6 +43,7 @@ struct BwdParams {
     const float* lse;    // [Hq, T]
     const float* delta;  // [Hq, T]
     float* dq_acc;       // [Hq, T, D] fp32 (head-major; D = the kernel's padded head dimension)
+    int* dq_turn;        // [Hq, T] turn counters of the deterministic mode (null otherwise), zeroed per call
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     int* status;
@@ -80,14 +81,14 @@ struct BwdCfg {
 
 enum BwdSite {
     kBSiteKvFull = 21, kBSiteQFull = 22, kBSiteQEmpty = 23, kBSiteSFull = 24, kBSiteDpFull = 25, kBSitePReady = 26,
-    kBSiteDsReady = 27, kBSiteDsFree = 28, kBSiteDqFull = 29, kBSiteDqEmpty = 30, kBSiteDkvFull = 31, kBSiteDrain = 32
+    kBSiteDsReady = 27, kBSiteDsFree = 28, kBSiteDqFull = 29, kBSiteDqEmpty = 30, kBSiteDkvFull = 31, kBSiteDrain = 32, kBSiteTurn = 33
 };
 
 template <int D>
 __global__ void __launch_bounds__(256)
 sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ dout,
-                           float* __restrict__ delta, float* __restrict__ dq_acc, int T, int Hq, int d,
-                           const TensorLayout lay) {
+                           float* __restrict__ delta, float* __restrict__ dq_acc, int* __restrict__ dq_turn, int T,
+                           int Hq, int d, const TensorLayout lay) {
     constexpr int kLanesPerRow = D / 8;
     const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     const long long row = gid / kLanesPerRow;  // row = global token * Hq + head
@@ -123,6 +124,7 @@ sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloa
         const long long tok = row / Hq;
         const int h = static_cast<int>(row % Hq);
         delta[static_cast<long long>(h) * T + tok] = acc;
+        if (dq_turn != nullptr) dq_turn[static_cast<long long>(h) * T + tok] = 0;
     }
 }
 
@@ -180,13 +182,18 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // causal: low key tiles see the most query tiles -> launch them first
     const int n_tiles_grid = static_cast<int>(gridDim.x) / p.group_chunk;
     const int jt_raw = static_cast<int>(blockIdx.x) / p.group_chunk;
-    const int jt = p.causal ? jt_raw : n_tiles_grid - 1 - jt_raw;
+    // The deterministic mode launches the high (light) key tiles first, so that a tile only ever waits for
+    // tiles launched before it (see the turn counters in the reduction group).
+    const int jt = (p.causal && p.dq_turn == nullptr) ? jt_raw : n_tiles_grid - 1 - jt_raw;
     const int kv0 = jt * 128;
     if (kv0 >= L) return;
     const int n_qs = (L + 63) >> 6;            // 64-row query steps in the sequence
     const int i_start = p.causal ? 2 * jt : 0;  // first query step that sees this key tile
     const int per_head = n_qs - i_start;
     const int n_it = G * per_head;
+    const bool det = p.dq_turn != nullptr;
+    const int nt_seq = (L + 127) >> 7;  // key tiles of this sequence
+    auto step_of = [&](int it) { return i_start + it % per_head; };
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = smem_raw;
@@ -277,7 +284,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         uint32_t stage = wg % NS, sphase = 0;
         for (int s = wg; s < n_it && ok; s += 2) {
             const uint32_t ph = (s >> 1) & 1;
-            const int q0 = (i_start + s % per_head) * 64;
+            const int q0 = step_of(s) * 64;
             const bool need_mask = (p.causal && q0 < kv0 + 128) || (kv0 + 128 > L);
             // rows (lse * log2e, D_i) of this step were staged by the producer warp together with Q / dO
             if (r == 0) SDPA_TR(0, s, 0);
@@ -417,9 +424,18 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int x = tid & 127;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         bool ok = true;
+        // Deterministic mode: the key tiles that see a query step add into it from the highest tile index
+        // down.  That is the order in which they reach the step anyway (tile j starts its sweep at step 2j
+        // under a causal mask), and the tiles waited for were launched earlier.  The counter of a step holds
+        // how many tiles have added.  Thread 32 waits for this tile's rank while the group stages the step;
+        // thread 0 adds and passes the turn on two steps later, when `cp.async.bulk.wait_group 2` says that
+        // the adds have been performed: their latency (L2 reduce throughput plus a round trip) is longer
+        // than one step.  A wait that gives up raises the CTA's abort flag; the adds are then skipped.
+        int* pend_turn[2] = {nullptr, nullptr};  // thread 0: turns of the last two steps, oldest first
+        int pend_val[2] = {0, 0};
         for (int it = 0; it < n_it && ok; ++it) {
             const int h = g * G + it / per_head;
-            const int q0 = (i_start + it % per_head) * 64;
+            const int q0 = step_of(it) * 64;
             if (x == 0) SDPA_TR(4, it, 0);
             ok = mbar_wait_warp(&dq_full[it & 1], (it >> 1) & 1, ctl, kBSiteDqFull);
             if (!ok) break;
@@ -433,6 +449,24 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tc_fence_before();
             mbar_arrive(&dq_empty[it & 1]);
             if (x == 0) SDPA_TR(4, it, 2);
+            int* turn = nullptr;
+            int rank = 0;
+            if (det) {
+                const int j_last = p.causal ? min(nt_seq - 1, (q0 + 63) >> 7) : nt_seq - 1;  // highest tile on this step
+                rank = j_last - jt;
+                turn = p.dq_turn + static_cast<size_t>(h) * p.T + sp.gt0 + q0;
+                if (x == 32) wait_turn(turn, rank, ctl, kBSiteTurn);  // sets the abort flag on failure
+                if (x == 0 && pend_turn[0] != nullptr) {
+                    bulk_wait<2>();  // all but the previous step's two groups: the adds of two steps ago are done
+                    SDPA_TR(4, it, 6);
+                    if (!*ctl.abort) release_turn(pend_turn[0], pend_val[0]);
+                    SDPA_TR(4, it, 7);
+                }
+                if (x == 0) {
+                    pend_turn[0] = pend_turn[1]; pend_val[0] = pend_val[1];
+                    pend_turn[1] = turn;         pend_val[1] = rank + 1;
+                }
+            }
             // Two halves of 32 query rows, each its own bulk group: the rows of one half are rewritten
             // while the bulk engine is still reading the other half of the previous step.
             const int nq = min(64, L - q0);
@@ -451,7 +485,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (x == 0) {
                     const int rows = min(32, nq - hf * 32);
 #ifndef SDPA_EXP_NO_REDUCE
-                    if (rows > 0)
+                    if (rows > 0 && !(det && *ctl.abort))
                         bulk_reduce_add_f32(dst + hf * 32 * D, sDQ + hf * 32 * D, static_cast<uint32_t>(rows) * D * 4u);
 #endif
                     bulk_commit();  // committed even when empty, so the group count per step is fixed
@@ -461,7 +495,13 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (x == 0) SDPA_TR(4, it, 4);
             if (x == 0) SDPA_TR(4, it, 5);
         }
-        if (x == 0) bulk_wait<0>();
+        if (x == 0) {
+            bulk_wait<0>();
+            if (det && !*ctl.abort) {
+                if (pend_turn[0] != nullptr) release_turn(pend_turn[0], pend_val[0]);
+                if (pend_turn[1] != nullptr) release_turn(pend_turn[1], pend_val[1]);
+            }
+        }
     } else if (warp == 13) {
         // ------------------------------------------------------------ producer warp (all 32 lanes)
         // Lane 0 issues the TMA loads; every lane stages two (lse * log2e, D_i) pairs of the step's 64
@@ -482,7 +522,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             ok = mbar_wait_warp(&q_empty[st], ph ^ 1, ctl, kBSiteQEmpty);
             if (!ok) break;
             const int h = g * G + it / per_head;
-            const int q0 = (i_start + it % per_head) * 64;
+            const int q0 = step_of(it) * 64;
             if (lane == 0) {
                 uint8_t* dst = sQdO + st * Cfg::kStageBytes;
                 mbar_arrive_expect_tx(&q_full[st], Cfg::kStageBytes);

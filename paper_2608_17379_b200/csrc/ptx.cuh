@@ -96,6 +96,34 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, c
     return __all_sync(0xffffffffu, ok);
 }
 
+// Bounded wait until a global int reaches `want` (acquire loads).  Used for the turn counters that order
+// the dQ accumulation of the deterministic backward mode; the value is written by an earlier-launched CTA.
+__device__ __forceinline__ bool wait_turn(const int* sem, int want, const WaitCtl& ctl, int site) {
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    for (;;) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(sem) : "memory");
+        if (v == want) return true;
+        if ((++spins & 15u) == 0u) {
+            if (*ctl.abort) return false;
+            if (clock64() - t0 > ctl.limit) {
+                *ctl.abort = 1;
+                atomicCAS(ctl.g_status, 0, (site << 8) | kStatusTimeout);
+                return false;
+            }
+        }
+    }
+}
+// Passes a turn on.  The caller has waited (cp.async.bulk.wait_group) until its bulk reduce-adds were
+// performed, so they are in the L2, the point every later reduce-add of any SM goes through; the counter
+// only has to be written after that.  A gpu-scope release store was measured at about 1.2 k cycles here
+// and is not needed for that ordering; the proxy fence orders the async-proxy writes before this store.
+__device__ __forceinline__ void release_turn(int* sem, int value) {
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(sem), "r"(value) : "memory");
+}
+
 // ------------------------------------------------------------------ fences / misc
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -314,13 +314,14 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
 extern "C" size_t sdpa_bwd_workspace_bytes(int B, int Hq, int Hkv, int D, int total_tokens, int max_seqlen) {
     if (B < 1 || Hq < 1 || Hkv < 1 || total_tokens < 0 || max_seqlen < 0 || D < 8 || D > 128 || (D % 8) != 0 || Hq % Hkv != 0)
         return 0;
-    return bwd_dq_bytes(Hq, padded_head_dim(D), total_tokens) + bwd_delta_bytes(Hq, total_tokens) + 256;
+    // fp32 dQ accumulator, D_i rows, turn counters of the deterministic mode (same size as the D_i rows)
+    return bwd_dq_bytes(Hq, padded_head_dim(D), total_tokens) + 2 * bwd_delta_bytes(Hq, total_tokens) + 256;
 }
 
 static int bwd_launch(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
                       void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D,
                       int causal, float scale, int total_tokens, int max_seqlen, void* workspace,
-                      size_t workspace_bytes, void* stream, const TensorLayout& lay) {
+                      size_t workspace_bytes, void* stream, const TensorLayout& lay, bool deterministic = false) {
     int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen, lay.dense != 0);
     if (rc != SDPA_OK) return rc;
     if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
@@ -339,6 +340,8 @@ static int bwd_launch(const void* q, const void* k, const void* v, const void* o
     float* dq_acc = static_cast<float*>(workspace);
     const int Dp = padded_head_dim(D);
     float* delta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + bwd_dq_bytes(Hq, Dp, total_tokens));
+    int* dq_turn = deterministic ? reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(delta) + bwd_delta_bytes(Hq, total_tokens))
+                                 : nullptr;
 
     // B0: D_i = rowsum(dO * O), and clear the fp32 dQ accumulator.
     {
@@ -348,11 +351,11 @@ static int bwd_launch(const void* q, const void* k, const void* v, const void* o
         const long long blocks = (rows + rows_per_block - 1) / rows_per_block;
         if (Dp == 128)
             sdpa_bwd_preprocess_kernel<128><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
-                static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
+                static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc, dq_turn,
                 total_tokens, Hq, D, lay);
         else
             sdpa_bwd_preprocess_kernel<64><<<static_cast<unsigned>(blocks), threads, 0, s>>>(
-                static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc,
+                static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), delta, dq_acc, dq_turn,
                 total_tokens, Hq, D, lay);
         SDPA_CUDA_TRY(cudaGetLastError());
     }
@@ -370,6 +373,7 @@ static int bwd_launch(const void* q, const void* k, const void* v, const void* o
     p.lse = lse;
     p.delta = delta;
     p.dq_acc = dq_acc;
+    p.dq_turn = dq_turn;
     p.dk = static_cast<__nv_bfloat16*>(dk);
     p.dv = static_cast<__nv_bfloat16*>(dv);
     p.status = st->status_ptr;
@@ -413,6 +417,14 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
                         size_t workspace_bytes, void* stream) {
     return bwd_launch(q, k, v, o, lse, dout, dq, dk, dv, cu_seqlens, B, Hq, Hkv, D, causal, scale, total_tokens,
                       max_seqlen, workspace, workspace_bytes, stream, packed_layout(total_tokens, Hq, Hkv, D));
+}
+
+extern "C" int sdpa_bwd_deterministic(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                                      const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B,
+                                      int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
+                                      void* workspace, size_t workspace_bytes, void* stream) {
+    return bwd_launch(q, k, v, o, lse, dout, dq, dk, dv, cu_seqlens, B, Hq, Hkv, D, causal, scale, total_tokens,
+                      max_seqlen, workspace, workspace_bytes, stream, packed_layout(total_tokens, Hq, Hkv, D), true);
 }
 
 extern "C" int sdpa_bwd_bhsd(const void* q, const void* k, const void* v, const void* o, const float* lse,
