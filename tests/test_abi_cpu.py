@@ -66,6 +66,18 @@ def test_argument_checks_come_before_any_cuda_call(lib):
     assert bwd(a, need - 1) == -4
     assert bwd(a + 16, need) == -4
     assert lib.sdpa_host_staging_bytes(1, 2, 2, 64, 8, 8) > need
+    det = lambda ws, n: lib.sdpa_bwd_deterministic(a, a, a, a, a, a, a, a, a, a, 1, 2, 2, 64, 0, 1.0, 8, 8, ws, n, None)
+    assert det(None, need) == -4 and det(a, need - 1) == -4
+    # dense [B, H, S, D] entry points: cu_seqlens is optional, the other checks are the same
+    fd = lambda **kw: lib.sdpa_fwd_bhsd(kw.get("q", a), a, a, a, a, kw.get("cu", None), kw.get("B", 1), kw.get("Hq", 2),
+                                        kw.get("Hkv", 2), kw.get("S", 8), kw.get("D", 64), 0, kw.get("scale", 1.0), None)
+    assert fd(q=None) == -1
+    assert fd(q=a + 2) == -2
+    assert fd(D=100) == -3 and fd(Hq=3, Hkv=2) == -3 and fd(B=0) == -3 and fd(S=-1) == -3
+    assert fd(B=1 << 20, S=1 << 20) == -3      # B * S must fit 32 bits
+    assert fd(S=0) == 0                        # empty sequences: valid no-op
+    bd = lambda ws, n: lib.sdpa_bwd_bhsd(a, a, a, a, a, a, a, a, a, None, 1, 2, 2, 8, 64, 0, 1.0, ws, n, None)
+    assert bd(None, need) == -4 and bd(a, need - 1) == -4
 
 
 def test_no_silent_fallback_without_a_gpu(lib):
