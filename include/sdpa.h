@@ -117,6 +117,30 @@ int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Forward and backward passes for sequences whose keys are not the rows of their queries (the paper's paged
+ * prefill workload has more keys than queries per sequence, appendix "Generalization attention workloads";
+ * these are the same operator on packed tensors, with its backward pass):
+ *        q, o, dout, dq : bf16 [total_q, Hq,  D]     rows of sequence b: cu_seqlens_q[b] .. cu_seqlens_q[b+1]-1
+ *        k, v, dk, dv   : bf16 [total_k, Hkv, D]     rows of sequence b: cu_seqlens_k[b] .. cu_seqlens_k[b+1]-1
+ *        lse            : fp32 [Hq, total_q]
+ * causal != 0: query i of Lq attends to keys 0 .. i + (Lk - Lq) of its sequence (the last query sees the
+ * last key), which needs Lk >= Lq; causal == 0: to all Lk keys, which needs Lk >= 1 wherever Lq >= 1.  A
+ * sequence that breaks these rules is reported as SDPA_STATUS_BAD_CU_SEQLENS.  Keys of a sequence without
+ * queries get zero dk and dv.  max_seqlen_q / max_seqlen_k bound the query / key lengths and size the
+ * grids; the backward workspace is sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, total_q, max_seqlen_q).
+ * Everything else is as for sdpa_fwd / sdpa_bwd.
+ */
+int sdpa_fwd_varlen_qk(const void* q, const void* k, const void* v, void* o, float* lse,
+                       const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k, int B, int Hq, int Hkv,
+                       int D, int causal, float scale, int total_q, int total_k, int max_seqlen_q,
+                       int max_seqlen_k, void* stream);
+int sdpa_bwd_varlen_qk(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                       const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens_q,
+                       const int32_t* cu_seqlens_k, int B, int Hq, int Hkv, int D, int causal,
+                       float scale, int total_q, int total_k, int max_seqlen_q, int max_seqlen_k,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * sdpa_bwd with a reproducible dq (the paper's backward workloads do not ask for this; the libraries it
  * compares with offer such a mode).  sdpa_bwd adds the dq contributions of the key tiles of a sequence
  * with fp32 reduce-adds in whatever order the tiles get there, so the last bits of dq can differ from run

@@ -19,7 +19,7 @@ SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
            "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout", "sdpa_fwd_paged",
-           "sdpa_fwd_bhsd", "sdpa_bwd_bhsd", "sdpa_bwd_deterministic")
+           "sdpa_fwd_bhsd", "sdpa_bwd_bhsd", "sdpa_bwd_deterministic", "sdpa_fwd_varlen_qk", "sdpa_bwd_varlen_qk")
 
 
 class SdpaError(RuntimeError):
@@ -42,6 +42,10 @@ def load():
     lib.sdpa_bwd_workspace_bytes.argtypes = [ci] * 6
     lib.sdpa_bwd.restype = ci
     lib.sdpa_bwd.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, cf, ci, ci, vp, ctypes.c_size_t, vp]
+    lib.sdpa_fwd_varlen_qk.restype = ci
+    lib.sdpa_fwd_varlen_qk.argtypes = [vp] * 7 + [ci, ci, ci, ci, ci, cf, ci, ci, ci, ci, vp]
+    lib.sdpa_bwd_varlen_qk.restype = ci
+    lib.sdpa_bwd_varlen_qk.argtypes = [vp] * 11 + [ci, ci, ci, ci, ci, cf, ci, ci, ci, ci, vp, ctypes.c_size_t, vp]
     lib.sdpa_bwd_deterministic.restype = ci
     lib.sdpa_bwd_deterministic.argtypes = lib.sdpa_bwd.argtypes
     lib.sdpa_host_staging_bytes.restype = ctypes.c_size_t
@@ -142,6 +146,44 @@ def sdpa_bwd(q, k, v, o, lse, dout, cu_seqlens, max_seqlen: int, causal: bool, s
             _ptr(cu_seqlens), B, Hq, Hkv, D, int(bool(causal)), float(scale), T, int(max_seqlen),
             _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
     _check(rc, "sdpa_bwd_deterministic" if deterministic else "sdpa_bwd")
+    return dq, dk, dv
+
+
+def sdpa_fwd_varlen_qk(q, k, v, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, causal: bool,
+                       scale: float, o=None, lse=None, stream=None):
+    """Separate key lengths: q [Tq,Hq,D], k,v [Tk,Hkv,D]; end-aligned causal mask.  Returns (o, lse [Hq,Tq])."""
+    lib = load()
+    Tq, Hq, Hkv, D = q.shape[0], q.shape[1], k.shape[1], q.shape[2]
+    assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and q.dtype == torch.bfloat16
+    B = cu_seqlens_q.numel() - 1
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((Hq, Tq), dtype=torch.float32, device=q.device)
+    rc = lib.sdpa_fwd_varlen_qk(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(cu_seqlens_q), _ptr(cu_seqlens_k),
+                                B, Hq, Hkv, D, int(bool(causal)), float(scale), Tq, k.shape[0], int(max_seqlen_q),
+                                int(max_seqlen_k), _stream_ptr(stream))
+    _check(rc, "sdpa_fwd_varlen_qk")
+    return o, lse
+
+
+def sdpa_bwd_varlen_qk(q, k, v, o, lse, dout, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int,
+                       causal: bool, scale: float, dq=None, dk=None, dv=None, workspace=None, stream=None):
+    """Gradients for sdpa_fwd_varlen_qk."""
+    lib = load()
+    Tq, Hq, Hkv, D = q.shape[0], q.shape[1], k.shape[1], q.shape[2]
+    B = cu_seqlens_q.numel() - 1
+    need = sdpa_bwd_workspace_bytes(B, Hq, Hkv, D, Tq, int(max_seqlen_q))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    rc = lib.sdpa_bwd_varlen_qk(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk),
+                                _ptr(dv), _ptr(cu_seqlens_q), _ptr(cu_seqlens_k), B, Hq, Hkv, D, int(bool(causal)),
+                                float(scale), Tq, k.shape[0], int(max_seqlen_q), int(max_seqlen_k), _ptr(workspace),
+                                int(workspace.numel()), _stream_ptr(stream))
+    _check(rc, "sdpa_bwd_varlen_qk")
     return dq, dk, dv
 
 

@@ -40,6 +40,8 @@ __device__ long long g_trace[5 * 32 * 8];
 
 struct BwdParams {
     const int32_t* cu_seqlens;
+    const int32_t* cu_seqlens_k;  // key rows of sequence b in k / v / dk / dv (packed layout), or null: the query rows
+    int Tk;                       // rows of k / v when cu_seqlens_k is given
     const float* lse;    // [Hq, T]
     const float* delta;  // [Hq, T]
     float* dq_acc;       // [Hq, T, D] fp32 (head-major; D = the kernel's padded head dimension)
@@ -186,13 +188,37 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // tiles launched before it (see the turn counters in the reduction group).
     const int jt = (p.causal && p.dq_turn == nullptr) ? jt_raw : n_tiles_grid - 1 - jt_raw;
     const int kv0 = jt * 128;
-    if (kv0 >= L) return;
+    // Keys of the sequence: the rows of its queries, or a row range of their own with Lk keys for L queries;
+    // a causal query i then sees keys 0 .. i + off, off = Lk - L (the last query sees the last key).
+    int rk0 = r0, Lk = L;
+    if (p.cu_seqlens_k != nullptr) {
+        rk0 = p.cu_seqlens_k[b];
+        const int rk1 = p.cu_seqlens_k[b + 1];
+        Lk = rk1 - rk0;
+        if (rk0 < 0 || rk1 > p.Tk || Lk < 0 || (L > 0 && (Lk < 1 || (p.causal && Lk < L)))) {
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
+            return;
+        }
+    }
+    const int off = Lk - L;
+    if (kv0 >= Lk) return;
+    if (L == 0) {
+        // keys without any query: their gradients are zero (only possible with separate key lengths)
+        const int rows = min(128, Lk - kv0), d8 = p.d >> 3;
+        for (int i = threadIdx.x; i < rows * d8; i += blockDim.x) {
+            const long long o8 = static_cast<long long>(rk0 + kv0 + i / d8) * p.lay.ts_kv +
+                                 static_cast<long long>(g) * p.lay.hs_kv + (i % d8) * 8;
+            *reinterpret_cast<uint4*>(p.dk + o8) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(p.dv + o8) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        return;
+    }
     const int n_qs = (L + 63) >> 6;            // 64-row query steps in the sequence
-    const int i_start = p.causal ? 2 * jt : 0;  // first query step that sees this key tile
+    const int i_start = p.causal ? max(0, kv0 - off) >> 6 : 0;  // first query step that sees this key tile
     const int per_head = n_qs - i_start;
     const int n_it = G * per_head;
     const bool det = p.dq_turn != nullptr;
-    const int nt_seq = (L + 127) >> 7;  // key tiles of this sequence
+    const int nt_seq = (Lk + 127) >> 7;  // key tiles of this sequence
     auto step_of = [&](int it) { return i_start + it % per_head; };
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -275,7 +301,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int wg = warp >> 2;
         const int r = tid & 127;           // key row inside the tile
         const int key = kv0 + r;           // key index inside the sequence
-        const bool key_ok = key < L;
+        const bool key_ok = key < Lk;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_base + kColS + wg * 64;
         const uint32_t tDP = tmem + lane_base + kColDP + wg * 64;
@@ -285,7 +311,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int s = wg; s < n_it && ok; s += 2) {
             const uint32_t ph = (s >> 1) & 1;
             const int q0 = step_of(s) * 64;
-            const bool need_mask = (p.causal && q0 < kv0 + 128) || (kv0 + 128 > L);
+            const bool need_mask = (p.causal && q0 + off < kv0 + 128) || (kv0 + 128 > Lk);
             // rows (lse * log2e, D_i) of this step were staged by the producer warp together with Q / dO
             if (r == 0) SDPA_TR(0, s, 0);
             ok = mbar_wait_warp(&q_full[stage], sphase, ctl, kBSiteQFull);
@@ -313,7 +339,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         float v = fast_exp2(fmaf(__uint_as_float(sr[i]), p.scale_log2, -lv[e]));
                         if (need_mask) {
                             const int qq = q0 + c * 32 + i;
-                            if (!key_ok || (p.causal && key > qq)) v = 0.f;
+                            if (!key_ok || (p.causal && key > qq + off)) v = 0.f;
                         }
                         pr[c * 32 + i] = v;
                     }
@@ -402,14 +428,14 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             {
                 const int lane = tid & 31;
                 const int k = lane % kChunks;
-                const int rows_left = L - kv0;  // keys of this tile inside the sequence
+                const int rows_left = Lk - kv0;  // keys of this tile inside the sequence
 #pragma unroll
                 for (int pass = 0; pass < 32 / kRowsPerPass; ++pass) {
                     const int rr = (warp & 3) * 32 + pass * kRowsPerPass + lane / kChunks;
                     if (rr < rows_left && k * 8 < p.d) {
                         const uint4 w = *reinterpret_cast<const uint4*>(out_stage + rr * (D * 2) + ((k ^ (rr & 7)) << 4));
                         __nv_bfloat16* dst = out + sp.bidx * p.lay.bs_kv +
-                                             static_cast<long long>(r0 + kv0 + rr) * p.lay.ts_kv +
+                                             static_cast<long long>(rk0 + kv0 + rr) * p.lay.ts_kv +
                                              static_cast<long long>(g) * p.lay.hs_kv;
                         *reinterpret_cast<uint4*>(dst + k * 8) = w;
                     }
@@ -452,7 +478,7 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             int* turn = nullptr;
             int rank = 0;
             if (det) {
-                const int j_last = p.causal ? min(nt_seq - 1, (q0 + 63) >> 7) : nt_seq - 1;  // highest tile on this step
+                const int j_last = p.causal ? min(nt_seq - 1, (q0 + 63 + off) >> 7) : nt_seq - 1;  // highest tile on this step
                 rank = j_last - jt;
                 turn = p.dq_turn + static_cast<size_t>(h) * p.T + sp.gt0 + q0;
                 if (x == 32) wait_turn(turn, rank, ctl, kBSiteTurn);  // sets the abort flag on failure
@@ -511,8 +537,8 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             mbar_arrive_expect_tx(kv_full, 2 * Cfg::kTileBytes);
 #pragma unroll
             for (int a = 0; a < D / 64; ++a) {
-                SDPA_TMA_LOAD_ROWS(sK + a * Cfg::kAtomBytes, &map_k, kv_full, a * 64, r0 + kv0, g, sp.bidx, p.lay.dense);
-                SDPA_TMA_LOAD_ROWS(sV + a * Cfg::kAtomBytes, &map_v, kv_full, a * 64, r0 + kv0, g, sp.bidx, p.lay.dense);
+                SDPA_TMA_LOAD_ROWS(sK + a * Cfg::kAtomBytes, &map_k, kv_full, a * 64, rk0 + kv0, g, sp.bidx, p.lay.dense);
+                SDPA_TMA_LOAD_ROWS(sV + a * Cfg::kAtomBytes, &map_v, kv_full, a * 64, rk0 + kv0, g, sp.bidx, p.lay.dense);
             }
         }
         bool ok = true;

@@ -26,6 +26,8 @@ namespace sdpa {
 
 struct FwdParams {
     const int32_t* cu_seqlens;   // query rows of sequence b: cu_seqlens[b] .. cu_seqlens[b+1]-1
+    const int32_t* cu_seqlens_k; // key rows of sequence b in k / v (packed layout), or null: same rows as the queries
+    int Tk;                      // rows of k / v when cu_seqlens_k is given
     // paged variant only: keys/values of sequence b are the cache rows kv_indices[kv_indptr[b] + j]
     const int32_t* kv_indptr;
     const int32_t* kv_indices;
@@ -80,9 +82,10 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// kPaged = false: K/V are packed [T, Hkv, D] tensors loaded by TMA, keys and queries of a sequence have
-// equal length.  kPaged = true: K/V rows are gathered from a page-size-1 cache through a page table,
-// a sequence may have more keys than queries, and a causal query i sees keys 0 .. i + (Lk - Lq).
+// kPaged = false: K/V are tensors loaded by TMA; the keys of a sequence are the rows of its queries, or (packed
+// layout, cu_seqlens_k given) a row range of their own.  kPaged = true: K/V rows are gathered from a
+// page-size-1 cache through a page table.  Whenever a sequence has Lk keys for Lq queries, a causal query i
+// sees keys 0 .. i + (Lk - Lq): the last query sees the last key.
 template <int D, bool kPaged>
 __global__ void __launch_bounds__(384, 1)
 sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -114,6 +117,18 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         kbase = p.kv_indptr[b];
         Lk = p.kv_indptr[b + 1] - kbase;
         if (Lk < L || kbase < 0) {  // fewer keys than queries would leave fully masked rows
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
+            return;
+        }
+    }
+    int rk0 = r0;  // first key row of the sequence in k / v
+    if (!kPaged && p.cu_seqlens_k != nullptr) {
+        rk0 = p.cu_seqlens_k[b];
+        const int rk1 = p.cu_seqlens_k[b + 1];
+        Lk = rk1 - rk0;
+        // every query row needs a visible key: at least one key, and under the end-aligned causal mask at
+        // least as many keys as queries
+        if (rk0 < 0 || rk1 > p.Tk || Lk < 1 || (p.causal && Lk < L)) {
             if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
             return;
         }
@@ -429,7 +444,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         ok = mbar_wait(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
                         if (!ok) break;
                         load_tile(kv == 0 ? &map_k : &map_v, sRing + st * Cfg::kTileBytes, &kv_full[st], g,
-                                  r0 + j * 128);
+                                  rk0 + j * 128);
                         if (j == 0 && kv == 0 && n_kv[1] > 0)
                             load_tile(&map_q, sQ + Cfg::kTileBytes, &q_full[1], h, r0 + q_start + 128);
                     }

@@ -189,11 +189,26 @@ static size_t bwd_delta_bytes(int Hq, int T) { return align_up(static_cast<size_
 
 using namespace sdpa;
 
+// Key side of a call whose sequences have their own key row ranges (packed layout only); cu == nullptr: the
+// keys of a sequence are the rows of its queries.
+struct KeySide {
+    const int32_t* cu = nullptr;
+    int total = 0;
+    int max_seqlen = 0;
+};
+static int check_key_side(const KeySide& ks, const TensorLayout& lay) {
+    if (ks.cu == nullptr) return SDPA_OK;
+    if (lay.dense) return SDPA_ERR_SHAPE;
+    if (ks.total < 0 || ks.max_seqlen < 0 || ks.max_seqlen > ks.total) return SDPA_ERR_SHAPE;
+    return SDPA_OK;
+}
+
 static int fwd_launch(const void* q, const void* k, const void* v, void* o, float* lse, const int32_t* cu_seqlens,
                       int B, int Hq, int Hkv, int D, int causal, float scale, int total_tokens, int max_seqlen,
-                      void* stream, const TensorLayout& lay) {
+                      void* stream, const TensorLayout& lay, const KeySide& ks = KeySide()) {
     int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen, lay.dense != 0);
     if (rc != SDPA_OK) return rc;
+    if ((rc = check_key_side(ks, lay)) != SDPA_OK) return rc;
     if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
     if (!q || !k || !v || !o || !lse) return SDPA_ERR_NULL;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || (reinterpret_cast<uintptr_t>(lse) & 3u))
@@ -204,13 +219,17 @@ static int fwd_launch(const void* q, const void* k, const void* v, void* o, floa
 
     CUtensorMap mq, mk, mv;
     const int map_rows = lay.dense ? lay.S : total_tokens;
+    const int key_rows = ks.cu != nullptr ? ks.total : map_rows;
+    if (key_rows == 0) return SDPA_ERR_SHAPE;  // queries without any key row
     if ((rc = make_map(&mq, q, lay, B, map_rows, Hq, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mk, k, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mv, v, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mk, k, lay, B, key_rows, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mv, v, lay, B, key_rows, Hkv, D, 128)) != SDPA_OK) return rc;
 
     FwdParams p;
     p.lay = lay;
     p.cu_seqlens = cu_seqlens;
+    p.cu_seqlens_k = ks.cu;
+    p.Tk = ks.total;
     p.kv_indptr = nullptr; p.kv_indices = nullptr; p.k_cache = nullptr; p.v_cache = nullptr; p.num_pages = 0;
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
@@ -223,7 +242,7 @@ static int fwd_launch(const void* q, const void* k, const void* v, void* o, floa
     p.scale_log2 = scale * 1.4426950408889634f;
     const int n_pairs = (max_seqlen + 255) / 256;
     if (n_pairs > 65535) return SDPA_ERR_SHAPE;
-    p.head_chunk = fwd_head_chunk(B, Hq, Hkv, D, total_tokens);
+    p.head_chunk = fwd_head_chunk(B, Hq, Hkv, D, key_rows);
     if (static_cast<long long>(n_pairs) * p.head_chunk > 0x7fffffffLL) return SDPA_ERR_SHAPE;
     dim3 grid(static_cast<unsigned>(n_pairs * p.head_chunk),
               static_cast<unsigned>((B * Hq + p.head_chunk - 1) / p.head_chunk), 1);
@@ -241,6 +260,17 @@ extern "C" int sdpa_fwd(const void* q, const void* k, const void* v, void* o, fl
                         void* stream) {
     return fwd_launch(q, k, v, o, lse, cu_seqlens, B, Hq, Hkv, D, causal, scale, total_tokens, max_seqlen, stream,
                       packed_layout(total_tokens, Hq, Hkv, D));
+}
+
+extern "C" int sdpa_fwd_varlen_qk(const void* q, const void* k, const void* v, void* o, float* lse,
+                                  const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k, int B, int Hq, int Hkv,
+                                  int D, int causal, float scale, int total_q, int total_k, int max_seqlen_q,
+                                  int max_seqlen_k, void* stream) {
+    if (cu_seqlens_k == nullptr) return SDPA_ERR_NULL;
+    KeySide ks;
+    ks.cu = cu_seqlens_k; ks.total = total_k; ks.max_seqlen = max_seqlen_k;
+    return fwd_launch(q, k, v, o, lse, cu_seqlens_q, B, Hq, Hkv, D, causal, scale, total_q, max_seqlen_q, stream,
+                      packed_layout(total_q, Hq, Hkv, D), ks);
 }
 
 // Limits of the dense entry points: B * S rows are indexed with 32-bit integers.
@@ -280,6 +310,8 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
     if ((rc = make_map(&mq, q, lay, 1, total_q, Hq, D, 128)) != SDPA_OK) return rc;
     FwdParams p;
     p.lay = lay;
+    p.cu_seqlens_k = nullptr;
+    p.Tk = 0;
     p.cu_seqlens = cu_seqlens_q;
     p.kv_indptr = kv_indptr;
     p.kv_indices = kv_indices;
@@ -321,11 +353,23 @@ extern "C" size_t sdpa_bwd_workspace_bytes(int B, int Hq, int Hkv, int D, int to
 static int bwd_launch(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
                       void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D,
                       int causal, float scale, int total_tokens, int max_seqlen, void* workspace,
-                      size_t workspace_bytes, void* stream, const TensorLayout& lay, bool deterministic = false) {
+                      size_t workspace_bytes, void* stream, const TensorLayout& lay, bool deterministic = false,
+                      const KeySide& ks = KeySide()) {
     int rc = check_common(cu_seqlens, B, Hq, Hkv, D, scale, total_tokens, max_seqlen, lay.dense != 0);
     if (rc != SDPA_OK) return rc;
-    if (total_tokens == 0 || max_seqlen == 0) return SDPA_OK;
+    if ((rc = check_key_side(ks, lay)) != SDPA_OK) return rc;
+    if (total_tokens == 0 || max_seqlen == 0) {
+        // no queries at all: keys that exist on their own get zero gradients
+        if (ks.cu != nullptr && ks.total > 0) {
+            if (!dk || !dv) return SDPA_ERR_NULL;
+            const size_t bytes = static_cast<size_t>(ks.total) * Hkv * D * 2;
+            SDPA_CUDA_TRY(cudaMemsetAsync(dk, 0, bytes, static_cast<cudaStream_t>(stream)));
+            SDPA_CUDA_TRY(cudaMemsetAsync(dv, 0, bytes, static_cast<cudaStream_t>(stream)));
+        }
+        return SDPA_OK;
+    }
     if (!q || !k || !v || !o || !lse || !dout || !dq || !dk || !dv) return SDPA_ERR_NULL;
+    if (ks.cu != nullptr && ks.total == 0) return SDPA_ERR_SHAPE;  // queries without any key row
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(dout) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || (reinterpret_cast<uintptr_t>(lse) & 3u))
         return SDPA_ERR_ALIGN;
@@ -362,14 +406,17 @@ static int bwd_launch(const void* q, const void* k, const void* v, const void* o
 
     CUtensorMap mq, mk, mv, mdo;
     const int map_rows = lay.dense ? lay.S : total_tokens;
+    const int key_rows = ks.cu != nullptr ? ks.total : map_rows;
     if ((rc = make_map(&mq, q, lay, B, map_rows, Hq, D, 64)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mk, k, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
-    if ((rc = make_map(&mv, v, lay, B, map_rows, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mk, k, lay, B, key_rows, Hkv, D, 128)) != SDPA_OK) return rc;
+    if ((rc = make_map(&mv, v, lay, B, key_rows, Hkv, D, 128)) != SDPA_OK) return rc;
     if ((rc = make_map(&mdo, dout, lay, B, map_rows, Hq, D, 64)) != SDPA_OK) return rc;
 
     BwdParams p;
     p.lay = lay;
     p.cu_seqlens = cu_seqlens;
+    p.cu_seqlens_k = ks.cu;
+    p.Tk = ks.total;
     p.lse = lse;
     p.delta = delta;
     p.dq_acc = dq_acc;
@@ -382,7 +429,7 @@ static int bwd_launch(const void* q, const void* k, const void* v, const void* o
     p.max_seqlen = max_seqlen;
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
-    const int n_kv_tiles = (max_seqlen + 127) / 128;
+    const int n_kv_tiles = ((ks.cu != nullptr ? ks.max_seqlen : max_seqlen) + 127) / 128;
     if (n_kv_tiles > 65535) return SDPA_ERR_SHAPE;
     // x walks a chunk of (sequence, kv head) groups key tile by key tile, y walks the chunks
     const int n_groups = B * Hkv;
@@ -417,6 +464,18 @@ extern "C" int sdpa_bwd(const void* q, const void* k, const void* v, const void*
                         size_t workspace_bytes, void* stream) {
     return bwd_launch(q, k, v, o, lse, dout, dq, dk, dv, cu_seqlens, B, Hq, Hkv, D, causal, scale, total_tokens,
                       max_seqlen, workspace, workspace_bytes, stream, packed_layout(total_tokens, Hq, Hkv, D));
+}
+
+extern "C" int sdpa_bwd_varlen_qk(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                                  const void* dout, void* dq, void* dk, void* dv, const int32_t* cu_seqlens_q,
+                                  const int32_t* cu_seqlens_k, int B, int Hq, int Hkv, int D, int causal, float scale,
+                                  int total_q, int total_k, int max_seqlen_q, int max_seqlen_k, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+    if (cu_seqlens_k == nullptr) return SDPA_ERR_NULL;
+    KeySide ks;
+    ks.cu = cu_seqlens_k; ks.total = total_k; ks.max_seqlen = max_seqlen_k;
+    return bwd_launch(q, k, v, o, lse, dout, dq, dk, dv, cu_seqlens_q, B, Hq, Hkv, D, causal, scale, total_q,
+                      max_seqlen_q, workspace, workspace_bytes, stream, packed_layout(total_q, Hq, Hkv, D), false, ks);
 }
 
 extern "C" int sdpa_bwd_deterministic(const void* q, const void* k, const void* v, const void* o, const float* lse,
