@@ -33,6 +33,8 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this same command on
 # the c3 workload (profiles/sdpa_kernels_c3_dram.md); null for other workloads.
 NCU_DRAM_TRAFFIC_C3 = {"sdpa_bwd_kernel<128>": 365212928 + 155866112, "sdpa_fwd_kernel<128>": 101782784 + 36194304}
+# sm__pipe_tensor_cycles_active.avg.pct_of_peak_sustained_active of the same capture (clock independent)
+NCU_TENSOR_ACTIVE_PCT_C3 = {"sdpa_bwd_kernel<128>": 57.76, "sdpa_fwd_kernel<128>": 58.01}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -407,9 +409,15 @@ def main():
                      "ms_per_launch": main_med, "flops_per_launch": w.bwd_flops(),
                      "traffic": NCU_DRAM_TRAFFIC_C3["sdpa_bwd_kernel<128>"] if w.name == "c3" else None,
                      "traffic_unit": "bytes per launch (ncu dram read+write)",
+                     "dram_gbs_at_traffic": (NCU_DRAM_TRAFFIC_C3["sdpa_bwd_kernel<128>"] / (main_med * 1e-3) / 1e9
+                                             if w.name == "c3" else None),
+                     "ncu_tensor_pipe_active_pct": (NCU_TENSOR_ACTIVE_PCT_C3["sdpa_bwd_kernel<128>"]
+                                                    if w.name == "c3" else None),
                      "fwd_kernel": {"kernel": "sdpa_fwd_kernel<128>", "achieved": fwd_tf, "frac": fwd_tf / peak,
                                     "ms_per_launch": fwd_ms, "flops_per_launch": w.fwd_flops(),
-                                    "traffic": NCU_DRAM_TRAFFIC_C3["sdpa_fwd_kernel<128>"] if w.name == "c3" else None},
+                                    "traffic": NCU_DRAM_TRAFFIC_C3["sdpa_fwd_kernel<128>"] if w.name == "c3" else None,
+                                    "ncu_tensor_pipe_active_pct": (NCU_TENSOR_ACTIVE_PCT_C3["sdpa_fwd_kernel<128>"]
+                                                                   if w.name == "c3" else None)},
                      "hbm_min_bytes_per_step": w.min_bytes_fwd() + w.min_bytes_bwd(),
                      "hbm_gbs_at_min_bytes": (w.min_bytes_fwd() + w.min_bytes_bwd()) / (step_ms * 1e-3) / 1e9,
                      "hbm_peak_gbs": float(peaks["hbm_gbs"])},
