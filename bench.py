@@ -31,7 +31,7 @@ from paper_2608_17379_b200 import workloads as W  # noqa: E402
 METRIC = "SDPA fwd+bwd TFLOPS (bf16, device-timed)"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this same command on
-# the c3 workload (profiles/sdpa_kernels_c3_dram.md); null for other workloads.
+# the c3 workload (its summary is kept under profiles/); null for other workloads.
 NCU_DRAM_TRAFFIC_C3 = {"sdpa_bwd_kernel<128>": 365212928 + 155866112, "sdpa_fwd_kernel<128>": 101782784 + 36194304}
 # sm__pipe_tensor_cycles_active.avg.pct_of_peak_sustained_active of the same capture (clock independent)
 NCU_TENSOR_ACTIVE_PCT_C3 = {"sdpa_bwd_kernel<128>": 57.76, "sdpa_fwd_kernel<128>": 58.01}

@@ -510,10 +510,8 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 named_bar_sync(2, 128);
                 if (x == 0) {
                     const int rows = min(32, nq - hf * 32);
-#ifndef SDPA_EXP_NO_REDUCE
                     if (rows > 0 && !(det && *ctl.abort))
                         bulk_reduce_add_f32(dst + hf * 32 * D, sDQ + hf * 32 * D, static_cast<uint32_t>(rows) * D * 4u);
-#endif
                     bulk_commit();  // committed even when empty, so the group count per step is fixed
                 }
                 if (x == 0 && hf == 0) SDPA_TR(4, it, 3);
