@@ -166,7 +166,8 @@ static int fwd_head_chunk(int B, int Hq, int Hkv, int D, long long kv_rows) {
     if (total <= kL2Budget || B <= 0) return all;
     const long long per_kv_head = std::max<long long>(1, kv_rows / B * D * 4);
     const long long kv_heads = std::max<long long>(1, kL2Budget / per_kv_head);
-    const long long chunk = kv_heads * (Hq / Hkv);
+    long long chunk = kv_heads * (Hq / Hkv);
+    chunk = std::max<long long>(chunk, (all + 65534) / 65535);  // the chunks are the grid's y dimension
     return static_cast<int>(std::min<long long>(all, chunk));
 }
 
@@ -177,7 +178,7 @@ static int fwd_head_chunk(int B, int Hq, int Hkv, int D, long long kv_rows) {
 static int bwd_group_chunk(int n_groups, int n_kv_tiles, long long dq_acc_bytes) {
     if (dq_acc_bytes <= (48ll << 20) || n_groups <= 8) return std::max(1, n_groups);
     const int c0 = std::max(8, (296 + n_kv_tiles - 1) / std::max(1, n_kv_tiles));
-    const int n_chunks = (n_groups + c0 - 1) / c0;
+    const int n_chunks = std::min((n_groups + c0 - 1) / c0, 65535);  // the chunks are the grid's y dimension
     return (n_groups + n_chunks - 1) / n_chunks;
 }
 

@@ -305,3 +305,13 @@ def test_d96_paper_shape_slices():
     and 8 heads so that the oracle checks every slice in seconds."""
     w = TL.random_workload((4096,), 8, 8, 96, True, seed=7196)
     run_and_compare(w, slices=[(0, 0), (0, 7)])
+
+
+def test_many_short_sequences():
+    """Two thousand sequences of 0..40 tokens (a decode-like batch): every CTA is a ragged tail, most grid
+    slots find nothing to do."""
+    rng = np.random.default_rng(77)
+    lengths = [int(x) for x in rng.integers(0, 41, 2000)]
+    w = TL.random_workload(lengths, 8, 2, 64, True, seed=7300)
+    slices = [(b, g) for b in range(0, 2000, 97) for g in range(2)]
+    run_and_compare(w, slices=slices)
