@@ -117,6 +117,26 @@ int sdpa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Decode over a paged KV cache (paper, appendix "Generalization attention workloads": GQA paged decode, one
+ * query token per sequence, page size 1).  The same operator as sdpa_fwd_paged with one query row per
+ * sequence, on a path built for that shape, which is bound by reading the K/V pages and not by arithmetic:
+ * a CTA owns one (sequence, kv head) and one split of its keys, the rows of its tile are the Hq / Hkv query
+ * heads of the group, so the group's pages are read once; a second small kernel merges the splits.
+ *        q, o    : bf16 [B, Hq, D]            (token b is the query of sequence b)
+ *        lse     : fp32 [Hq, B]
+ *        k_cache, v_cache, kv_indptr, kv_indices, num_pages : as for sdpa_fwd_paged
+ * The query sees all keys of its sequence; every sequence needs at least one key.  max_seqlen_k bounds the
+ * key count of a sequence and fixes the number of key splits.  `workspace` is caller-owned, 256-byte
+ * aligned device scratch of at least sdpa_decode_paged_workspace_bytes(...) bytes (fp32 partial results of
+ * the splits).  Hq / Hkv must not exceed 128.  Errors and status reporting as for sdpa_fwd_paged.
+ */
+size_t sdpa_decode_paged_workspace_bytes(int B, int Hq, int Hkv, int D, int max_seqlen_k);
+int sdpa_decode_paged(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                      const int32_t* kv_indptr, const int32_t* kv_indices, int B, int Hq, int Hkv, int D,
+                      float scale, int max_seqlen_k, int num_pages, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/*
  * Forward and backward passes for sequences whose keys are not the rows of their queries (the paper's paged
  * prefill workload has more keys than queries per sequence, appendix "Generalization attention workloads";
  * these are the same operator on packed tensors, with its backward pass):

@@ -19,7 +19,8 @@ SDPA_OK = 0
 EXPORTS = ("sdpa_fwd", "sdpa_bwd", "sdpa_bwd_workspace_bytes", "sdpa_query_status",
            "sdpa_status_string", "sdpa_last_cuda_error", "sdpa_host_staging_bytes",
            "sdpa_fwd_bwd_host", "sdpa_bwd_profile_events", "sdpa_bwd_static_scratch", "gemm_bf16_nt", "sdpa_selftest_wait_timeout", "sdpa_fwd_paged",
-           "sdpa_fwd_bhsd", "sdpa_bwd_bhsd", "sdpa_bwd_deterministic", "sdpa_fwd_varlen_qk", "sdpa_bwd_varlen_qk")
+           "sdpa_fwd_bhsd", "sdpa_bwd_bhsd", "sdpa_bwd_deterministic", "sdpa_fwd_varlen_qk", "sdpa_bwd_varlen_qk",
+           "sdpa_decode_paged", "sdpa_decode_paged_workspace_bytes")
 
 
 class SdpaError(RuntimeError):
@@ -46,6 +47,10 @@ def load():
     lib.sdpa_fwd_varlen_qk.argtypes = [vp] * 7 + [ci, ci, ci, ci, ci, cf, ci, ci, ci, ci, vp]
     lib.sdpa_bwd_varlen_qk.restype = ci
     lib.sdpa_bwd_varlen_qk.argtypes = [vp] * 11 + [ci, ci, ci, ci, ci, cf, ci, ci, ci, ci, vp, ctypes.c_size_t, vp]
+    lib.sdpa_decode_paged_workspace_bytes.restype = ctypes.c_size_t
+    lib.sdpa_decode_paged_workspace_bytes.argtypes = [ci] * 5
+    lib.sdpa_decode_paged.restype = ci
+    lib.sdpa_decode_paged.argtypes = [vp] * 7 + [ci, ci, ci, ci, cf, ci, ci, vp, ctypes.c_size_t, vp]
     lib.sdpa_bwd_deterministic.restype = ci
     lib.sdpa_bwd_deterministic.argtypes = lib.sdpa_bwd.argtypes
     lib.sdpa_host_staging_bytes.restype = ctypes.c_size_t
@@ -185,6 +190,28 @@ def sdpa_bwd_varlen_qk(q, k, v, o, lse, dout, cu_seqlens_q, cu_seqlens_k, max_se
                                 int(workspace.numel()), _stream_ptr(stream))
     _check(rc, "sdpa_bwd_varlen_qk")
     return dq, dk, dv
+
+
+def sdpa_decode_paged(q, k_cache, v_cache, kv_indptr, kv_indices, max_seqlen_k: int, scale: float, o=None,
+                      lse=None, workspace=None, stream=None):
+    """One query token per sequence over a page-size-1 cache: q [B,Hq,D], caches [P,Hkv,D].
+    Returns (o [B,Hq,D] bf16, lse [Hq,B] fp32)."""
+    lib = load()
+    B, Hq, D = q.shape
+    Hkv = k_cache.shape[1]
+    assert q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous() and q.dtype == torch.bfloat16
+    need = int(lib.sdpa_decode_paged_workspace_bytes(B, Hq, Hkv, D, int(max_seqlen_k)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((Hq, B), dtype=torch.float32, device=q.device)
+    rc = lib.sdpa_decode_paged(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(kv_indptr),
+                               _ptr(kv_indices), B, Hq, Hkv, D, float(scale), int(max_seqlen_k),
+                               int(k_cache.shape[0]), _ptr(workspace), int(workspace.numel()), _stream_ptr(stream))
+    _check(rc, "sdpa_decode_paged")
+    return o, lse
 
 
 def _dims_bhsd(q, k):

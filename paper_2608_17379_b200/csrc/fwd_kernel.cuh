@@ -42,6 +42,9 @@ struct FwdParams {
     int max_seqlen;
     int d;             // head dimension of the tensors (multiple of 8, <= D of the kernel; columns d..D-1 are zero padding)
     TensorLayout lay;  // strides of q / o (and of k / v for the non-paged kernel), lse
+    // decode variant only: per key split, unnormalised-free partial results of every (sequence, head)
+    float* part_o;     // [n_splits, B, Hq, d] fp32: softmax-weighted average of V over the split's keys
+    float* part_lse;   // [n_splits, B, Hq] fp32: log-sum-exp over the split's keys (-inf for an empty split)
     int head_chunk;    // (sequence, query head) pairs whose CTAs are launched interleaved
     float scale;       // softmax scale
     float scale_log2;  // scale * log2(e)
@@ -86,32 +89,50 @@ __device__ __forceinline__ void cp_async_wait() {
 // layout, cu_seqlens_k given) a row range of their own.  kPaged = true: K/V rows are gathered from a
 // page-size-1 cache through a page table.  Whenever a sequence has Lk keys for Lq queries, a causal query i
 // sees keys 0 .. i + (Lk - Lq): the last query sees the last key.
-template <int D, bool kPaged>
+template <int D, bool kPaged, bool kDecode = false>
 __global__ void __launch_bounds__(384, 1)
 sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
     using Cfg = FwdCfg<D>;
     constexpr int S = Cfg::kStages;
 
-    // Launch order: the (sequence, query head) pairs are taken in chunks of p.head_chunk; inside a chunk the
-    // CTAs go query-tile pair by pair (heaviest first), chunk after chunk, so the K/V rows that the CTAs
-    // running at one time walk through fit the L2 (the host picks the chunk from the K/V size per head).
-    const int bh = (int)blockIdx.y * p.head_chunk + (int)blockIdx.x % p.head_chunk;
-    if (bh >= p.B * p.Hq) return;
-    const int pair_raw = (int)blockIdx.x / p.head_chunk;
-    const int n_pairs_grid = (int)gridDim.x / p.head_chunk;
-    const int b = bh / p.Hq, h = bh % p.Hq;
-    const int g = h / (p.Hq / p.Hkv);
-    const int pair = n_pairs_grid - 1 - pair_raw;  // heaviest (latest) query tiles first
+    static_assert(!kDecode || kPaged, "the decode variant reads a paged cache");
+    int b, h, g, r0, L, q_start;
     SeqPos sp;
-    if (!locate_sequence(p.lay, p.cu_seqlens, b, p.T, p.max_seqlen, sp)) {
-        if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
-        return;
+    if (kDecode) {
+        // Decode: one query token per sequence.  A CTA owns one (sequence, kv head) and one split of its keys;
+        // the rows of its single query tile are the G query heads of the group (GQA packing), so the group's
+        // K/V rows are gathered once and not once per head.  grid = (B * Hkv, key splits).
+        const int bg = blockIdx.x;
+        b = bg / p.Hkv;
+        g = bg % p.Hkv;
+        h = g * (p.Hq / p.Hkv);  // first query head of the group
+        sp.tok0 = b; sp.bidx = 0; sp.gt0 = b; sp.L = 1;
+        r0 = b;
+        L = 1;
+        q_start = 0;
+    } else {
+        // Launch order: the (sequence, query head) pairs are taken in chunks of p.head_chunk; inside a chunk
+        // the CTAs go query-tile pair by pair (heaviest first), chunk after chunk, so the K/V rows that the
+        // CTAs running at one time walk through fit the L2 (the host picks the chunk from the K/V size per head).
+        const int bh = (int)blockIdx.y * p.head_chunk + (int)blockIdx.x % p.head_chunk;
+        if (bh >= p.B * p.Hq) return;
+        const int pair_raw = (int)blockIdx.x / p.head_chunk;
+        const int n_pairs_grid = (int)gridDim.x / p.head_chunk;
+        b = bh / p.Hq;
+        h = bh % p.Hq;
+        g = h / (p.Hq / p.Hkv);
+        const int pair = n_pairs_grid - 1 - pair_raw;  // heaviest (latest) query tiles first
+        if (!locate_sequence(p.lay, p.cu_seqlens, b, p.T, p.max_seqlen, sp)) {
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusBadCuSeqlens);
+            return;
+        }
+        r0 = sp.tok0;  // token coordinate of the sequence's first row
+        L = sp.L;
+        q_start = pair * 256;
+        if (q_start >= L) return;
     }
-    const int r0 = sp.tok0;  // token coordinate of the sequence's first row
-    const int L = sp.L;
-    const int q_start = pair * 256;
-    if (q_start >= L) return;
+    const int G = p.Hq / p.Hkv;
     int Lk = L, kbase = 0;  // number of keys of this sequence; first entry of its page list
     if (kPaged) {
         kbase = p.kv_indptr[b];
@@ -137,7 +158,18 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     int n_kv[2];
     const int n_kv_all = (Lk + 127) >> 7;
-    {
+    int tile_begin = 0;  // first key tile of this CTA (decode: the start of its split)
+    if (kDecode) {
+        const int per_split = (n_kv_all + (int)gridDim.y - 1) / (int)gridDim.y;
+        tile_begin = (int)blockIdx.y * per_split;
+        n_kv[0] = min(n_kv_all, tile_begin + per_split) - tile_begin;
+        n_kv[1] = 0;
+        if (n_kv[0] <= 0) {  // nothing in this split: the combining kernel skips a partial whose lse is -inf
+            if ((int)threadIdx.x < G)
+                p.part_lse[(static_cast<size_t>(blockIdx.y) * p.B + b) * p.Hq + h + threadIdx.x] = -INFINITY;
+            return;
+        }
+    } else {
         const bool has1 = (q_start + 128) < L;
         n_kv[0] = p.causal ? min(n_kv_all, ((q_start + 127 + off) >> 7) + 1) : n_kv_all;
         n_kv[1] = has1 ? (p.causal ? min(n_kv_all, ((q_start + 255 + off) >> 7) + 1) : n_kv_all) : 0;
@@ -200,7 +232,10 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int t = warp >> 2;                 // which query tile
         const int row_in_tile = tid & 127;
         const int row = q_start + t * 128 + row_in_tile;  // row inside the sequence
-        const bool valid = row < L;
+        const bool valid = kDecode ? row_in_tile < G : row < L;
+        // decode: only the first G rows of the tile are query heads; warps that own none of them do no
+        // arithmetic and only keep the barriers in step
+        const bool warp_live = !kDecode || (warp & 3) * 32 < G;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_base + t * 128;
         const uint32_t tO = tmem + lane_base + 256 + t * 128;
@@ -213,6 +248,12 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (!ok) break;
             if (row_in_tile == 0) SDPA_TR(t, j, 1);
             tc_fence_after();
+            if (!warp_live) {
+                tc_fence_before();
+                mbar_arrive(&p_half[t]);
+                mbar_arrive(&p_full[t]);
+                continue;
+            }
             float s[128];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -223,7 +264,11 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             tmem_wait_ld();
             if (row_in_tile == 0) SDPA_TR(t, j, 2);
-            const int key0 = j * 128;
+            if (kDecode && !valid) {  // rows past the group's heads hold whatever was in shared memory: neutralise them
+#pragma unroll
+                for (int c = 0; c < 128; ++c) s[c] = 0.f;
+            }
+            const int key0 = (tile_begin + j) * 128;
             const bool diag = p.causal && (key0 + 127 > q_start + t * 128 + off);
             if (diag || key0 + 128 > Lk) {
                 const int lim = p.causal ? min(row + off, Lk - 1) : (Lk - 1);  // last allowed key
@@ -309,7 +354,30 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (row_in_tile == 0) SDPA_TR(t, j, 5);
         }
         if (ok && n > 0) ok = mbar_wait_warp(&o_full[t], 0, ctl, kSiteOFull);
-        if (ok && n > 0) {
+        if (kDecode) {
+            // the G rows of the group leave as fp32 partial results of this key split
+            if (ok && n > 0 && warp_live) {
+                tc_fence_after();
+                const float inv_l = 1.0f / l;
+                const size_t slot = (static_cast<size_t>(blockIdx.y) * p.B + b) * p.Hq + h + row_in_tile;
+                float* dst = p.part_o + slot * p.d;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_x32(tO + c * 32, r);
+                    tmem_wait_ld();
+                    if (valid) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (c * 32 + i * 4 < p.d)
+                                *reinterpret_cast<float4*>(dst + c * 32 + i * 4) =
+                                    make_float4(__uint_as_float(r[4 * i]) * inv_l, __uint_as_float(r[4 * i + 1]) * inv_l,
+                                                __uint_as_float(r[4 * i + 2]) * inv_l, __uint_as_float(r[4 * i + 3]) * inv_l);
+                    }
+                }
+                if (valid) p.part_lse[slot] = m * p.scale + logf(l);
+            }
+        } else if (ok && n > 0) {
             tc_fence_after();
             const float inv_l = 1.0f / l;
             // O leaves through this tile's Q buffer (dead after the last S = Q K^T): every thread writes its
@@ -357,14 +425,18 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else {
         setmaxnreg_dec<80>();
-        if (warp == 9 && kPaged) {
-            // -------------------------------------------------------- gathering producer (all 32 lanes)
-            // Lane l copies key rows l, l+32, l+64, l+96 of each tile from the page-size-1 cache with
-            // 16-byte cp.async into the same 128B-swizzled layout a TMA load would produce; rows past
-            // the sequence end are zero-filled (a masked P of exactly 0 must not meet garbage in V).
+        if (warp >= 9 && kPaged) {
+            // -------------------------------------------------------- gathering producers (warps 9-11, all lanes)
+            // K_j is ring item 2j, V_j item 2j+1; item `it` is gathered by warp 9 + it % 3, so three tiles are
+            // in flight.  A tile's 128 rows come from the page-size-1 cache with 16-byte cp.async into the same
+            // 128B-swizzled layout a TMA load would produce; D/8 consecutive lanes copy one row (full lines in
+            // the cache), the page numbers travel by shuffle.  Rows past the sequence end and the padding
+            // columns are zero-filled (a masked P of exactly 0 must not meet garbage in V).
             const int lane = tid & 31;
-            if (lane == 0) {
-                mbar_arrive_expect_tx(&q_full[0], Cfg::kTileBytes);
+            const int pw = warp - 9;
+            if (pw == 0 && lane == 0) {
+                // decode: the Q map's box is the G heads of the group for one token (G rows of the tile)
+                mbar_arrive_expect_tx(&q_full[0], kDecode ? static_cast<uint32_t>(G) * D * 2u : Cfg::kTileBytes);
 #pragma unroll
                 for (int a = 0; a < D / 64; ++a)
                     SDPA_TMA_LOAD_ROWS(sQ + a * Cfg::kAtomBytes, &map_q, &q_full[0], a * 64, r0 + q_start, h, sp.bidx, p.lay.dense);
@@ -376,14 +448,17 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                     r0 + q_start + 128, h, sp.bidx, p.lay.dense);
                 }
             }
+            constexpr int kLanesPerRow = D / 8;               // 16-byte chunks of a row
+            constexpr int kRowsPerCopy = 32 / kLanesPerRow;    // rows one warp-wide cp.async covers
+            const int my_c = lane % kLanesPerRow;
+            const int my_sub = lane / kLanesPerRow;
             bool ok = true;
-            int it = 0;
-            int pending = -1;  // ring slot whose copies are in flight (one group deep)
-            for (int j = 0; j < n_iter && ok; ++j) {
-                int page[4];
+            for (int it = pw; it < 2 * n_iter && ok; it += 3) {
+                const int j = it >> 1, kv = it & 1;
+                int page[4];  // pages of the rows lane, lane+32, lane+64, lane+96 of key tile j (-1: past the end)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int key = j * 128 + lane + 32 * i;
+                    const int key = (tile_begin + j) * 128 + lane + 32 * i;
                     int pg = -1;
                     if (key < Lk) {
                         pg = p.kv_indices[kbase + key];
@@ -394,38 +469,29 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                     page[i] = pg;
                 }
-                for (int kv = 0; kv < 2 && ok; ++kv, ++it) {
-                    const int st = it % S;
-                    ok = mbar_wait_warp(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
-                    if (!ok) break;
-                    uint8_t* dst = sRing + st * Cfg::kTileBytes;
-                    const __nv_bfloat16* cache = kv == 0 ? p.k_cache : p.v_cache;
+                const int st = it % S;
+                ok = mbar_wait_warp(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
+                if (!ok) break;
+                uint8_t* dst = sRing + st * Cfg::kTileBytes;
+                const __nv_bfloat16* cache = kv == 0 ? p.k_cache : p.v_cache;
+                const bool col_real = my_c * 8 < p.d;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int row = lane + 32 * i;
-                        const bool have = page[i] >= 0;
-                        const __nv_bfloat16* src = cache + (static_cast<size_t>(have ? page[i] : 0) * p.Hkv + g) * p.d;
-#pragma unroll
-                        for (int c = 0; c < D / 8; ++c) {
-                            const bool real = have && c * 8 < p.d;  // padding columns and missing rows are zero-filled
-                            cp_async_16(dst + (c >> 3) * Cfg::kAtomBytes + sw128_offset(row, c & 7), real ? src + c * 8 : src,
-                                        real ? 16u : 0u);
-                        }
-                    }
-                    cp_async_commit();
-                    if (pending >= 0) {
-                        cp_async_wait<1>();          // the previous slot's copies have landed
-                        fence_proxy_async_smem();    // make them visible to the tensor core's reads
-                        mbar_arrive(&kv_full[pending]);
-                    }
-                    pending = st;
+                for (int rr = 0; rr < 128; rr += kRowsPerCopy) {
+                    const int row = rr + my_sub;
+                    const int pg = __shfl_sync(0xffffffffu, page[rr >> 5], row & 31);  // rr / 32 == row / 32
+                    const bool real = pg >= 0 && col_real;
+                    const __nv_bfloat16* src = cache + (static_cast<size_t>(pg >= 0 ? pg : 0) * p.Hkv + g) * p.d;
+                    cp_async_16(dst + (my_c >> 3) * Cfg::kAtomBytes + sw128_offset(row, my_c & 7), real ? src + my_c * 8 : src,
+                                real ? 16u : 0u);
                 }
+                cp_async_commit();
+                // The item is handed over before this warp asks for its next slot: that slot is freed by MMAs
+                // which may themselves be waiting for this item.  The overlap comes from the other two warps.
+                cp_async_wait<0>();          // the copies have landed
+                fence_proxy_async_smem();    // make them visible to the tensor core's reads
+                mbar_arrive(&kv_full[st]);
             }
             cp_async_wait<0>();
-            if (ok && pending >= 0) {
-                fence_proxy_async_smem();
-                mbar_arrive(&kv_full[pending]);
-            }
         } else if (warp == 9) {
             // -------------------------------------------------------- TMA producer
             if (elect_one()) {
@@ -563,6 +629,39 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_before();
     __syncthreads();
     if (warp == 8) tmem_dealloc(tmem, 512);
+}
+
+// Decode, second step: merges the key splits of every (sequence, head).  With lse_s the log-sum-exp and o_s
+// the softmax average of split s:  lse = log sum_s exp(lse_s),  o = sum_s exp(lse_s - lse) o_s.
+// One CTA per (sequence, head), one thread per 4 columns.
+__global__ void __launch_bounds__(32)
+sdpa_decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse,
+                           __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int n_splits, int B, int Hq, int d) {
+    const int bh = blockIdx.x;  // b * Hq + h
+    const int b = bh / Hq, h = bh % Hq;
+    const size_t stride = static_cast<size_t>(B) * Hq;
+    float mx = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, part_lse[s * stride + bh]);
+    float sum = 0.f;
+    for (int s = 0; s < n_splits; ++s) sum += expf(part_lse[s * stride + bh] - mx);
+    const float total = mx + logf(sum);
+    const int c = threadIdx.x * 4;
+    if (c < d) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < n_splits; ++s) {
+            const float ls = part_lse[s * stride + bh];
+            if (ls == -INFINITY) continue;  // empty split: its partial rows were never written
+            const float w = expf(ls - total);
+            const float4 v = *reinterpret_cast<const float4*>(part_o + (s * stride + bh) * d + c);
+            acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
+            acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+        }
+        uint2 w2;
+        w2.x = pack_bf16x2(acc.x, acc.y);
+        w2.y = pack_bf16x2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(o + static_cast<size_t>(bh) * d + c) = w2;
+    }
+    if (threadIdx.x == 0) lse[static_cast<size_t>(h) * B + b] = total;
 }
 
 }  // namespace sdpa

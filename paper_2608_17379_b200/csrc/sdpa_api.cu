@@ -80,6 +80,10 @@ static int device_state(DeviceState** out) {
                                                FwdCfg<128>::kSmemBytes));
             SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                FwdCfg<64>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               FwdCfg<128>::kSmemBytes));
+            SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_fwd_kernel<64, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               FwdCfg<64>::kSmemBytes));
             SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                BwdCfg<128>::kSmemBytes));
             SDPA_CUDA_TRY(cudaFuncSetAttribute(sdpa_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -97,18 +101,18 @@ static int device_state(DeviceState** out) {
 // Packed [T, H, D]: dims {D, H, T, 1}, box {64, 1, rows, 1}.  Dense [B, H, S, D]: dims {D, S, H, B}, box
 // {64, rows, 1, 1}.  Both keep the strides increasing and give the same [rows][64] tile in shared memory.
 static int make_map(CUtensorMap* map, const void* base, const TensorLayout& lay, int n_batch, int rows, int H, int D,
-                    int box_rows) {
+                    int box_rows, int box_heads = 1) {
     cuuint64_t dims[4], strides[3];
     cuuint32_t box[4];
     const cuuint64_t u = static_cast<cuuint64_t>(D) * 2;
     if (lay.dense) {
         dims[0] = D; dims[1] = rows; dims[2] = H; dims[3] = n_batch;
         strides[0] = u; strides[1] = u * rows; strides[2] = u * rows * H;
-        box[0] = 64; box[1] = box_rows; box[2] = 1; box[3] = 1;
+        box[0] = 64; box[1] = box_rows; box[2] = box_heads; box[3] = 1;
     } else {
         dims[0] = D; dims[1] = H; dims[2] = rows; dims[3] = 1;
         strides[0] = u; strides[1] = u * H; strides[2] = u * H * rows;
-        box[0] = 64; box[1] = 1; box[2] = box_rows; box[3] = 1;
+        box[0] = 64; box[1] = box_heads; box[2] = box_rows; box[3] = 1;
     }
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
@@ -231,6 +235,7 @@ static int fwd_launch(const void* q, const void* k, const void* v, void* o, floa
     p.cu_seqlens = cu_seqlens;
     p.cu_seqlens_k = ks.cu;
     p.Tk = ks.total;
+    p.part_o = nullptr; p.part_lse = nullptr;
     p.kv_indptr = nullptr; p.kv_indices = nullptr; p.k_cache = nullptr; p.v_cache = nullptr; p.num_pages = 0;
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
@@ -313,6 +318,7 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
     p.lay = lay;
     p.cu_seqlens_k = nullptr;
     p.Tk = 0;
+    p.part_o = nullptr; p.part_lse = nullptr;
     p.cu_seqlens = cu_seqlens_q;
     p.kv_indptr = kv_indptr;
     p.kv_indices = kv_indices;
@@ -340,6 +346,79 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
         sdpa_fwd_kernel<128, true><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mq, mq, p);
     else
         sdpa_fwd_kernel<64, true><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mq, mq, p);
+    SDPA_CUDA_TRY(cudaGetLastError());
+    return SDPA_OK;
+}
+
+// Key splits of the decode path: about two CTAs per SM of a B200 over all (sequence, kv head) pairs, at most
+// one split per 128-key tile of the longest sequence.
+static int decode_splits(int B, int Hkv, int max_seqlen_k) {
+    const long long groups = static_cast<long long>(B) * Hkv;
+    const int tiles = std::max(1, (max_seqlen_k + 127) / 128);
+    const long long want = (2 * 148 + groups - 1) / groups;
+    return static_cast<int>(std::max<long long>(1, std::min<long long>(want, tiles)));
+}
+
+extern "C" size_t sdpa_decode_paged_workspace_bytes(int B, int Hq, int Hkv, int D, int max_seqlen_k) {
+    if (B < 1 || Hq < 1 || Hkv < 1 || max_seqlen_k < 0 || D < 8 || D > 128 || (D % 8) != 0 || Hq % Hkv != 0) return 0;
+    const size_t rows = static_cast<size_t>(decode_splits(B, Hkv, max_seqlen_k)) * B * Hq;
+    return align_up(rows * D * sizeof(float), 256) + align_up(rows * sizeof(float), 256);
+}
+
+extern "C" int sdpa_decode_paged(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                                 const int32_t* kv_indptr, const int32_t* kv_indices, int B, int Hq, int Hkv, int D,
+                                 float scale, int max_seqlen_k, int num_pages, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+    if (B < 1 || Hq < 1 || Hkv < 1 || max_seqlen_k < 0 || num_pages < 0) return SDPA_ERR_SHAPE;
+    if (D < 8 || D > 128 || (D % 8) != 0 || Hq % Hkv != 0 || Hq / Hkv > 128) return SDPA_ERR_SHAPE;
+    if (!(scale > 0.f) || !isfinite(scale)) return SDPA_ERR_SHAPE;
+    if (!q || !k_cache || !v_cache || !o || !lse || !kv_indptr || !kv_indices) return SDPA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) ||
+        (reinterpret_cast<uintptr_t>(lse) & 3u))
+        return SDPA_ERR_ALIGN;
+    if (num_pages == 0 || max_seqlen_k == 0) return SDPA_ERR_SHAPE;  // every query needs at least one key
+    const size_t need = sdpa_decode_paged_workspace_bytes(B, Hq, Hkv, D, max_seqlen_k);
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
+        return SDPA_ERR_WORKSPACE;
+    DeviceState* st = nullptr;
+    int rc = device_state(&st);
+    if (rc != SDPA_OK) return rc;
+    const int G = Hq / Hkv;
+    const int n_splits = decode_splits(B, Hkv, max_seqlen_k);
+    const TensorLayout lay = packed_layout(B, Hq, Hkv, D);
+    CUtensorMap mq;  // box: the G heads of a group for one token
+    if ((rc = make_map(&mq, q, lay, 1, B, Hq, D, 1, G)) != SDPA_OK) return rc;
+    FwdParams p;
+    p.lay = lay;
+    p.cu_seqlens = nullptr; p.cu_seqlens_k = nullptr; p.Tk = 0;
+    p.kv_indptr = kv_indptr;
+    p.kv_indices = kv_indices;
+    p.k_cache = static_cast<const __nv_bfloat16*>(k_cache);
+    p.v_cache = static_cast<const __nv_bfloat16*>(v_cache);
+    p.num_pages = num_pages;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
+    p.status = st->status_ptr;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.T = B;
+    p.causal = 0;  // a single query token sees every key of its sequence
+    p.max_seqlen = 1;
+    p.d = D;
+    p.scale = scale;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.head_chunk = 1;
+    const size_t rows = static_cast<size_t>(n_splits) * B * Hq;
+    p.part_o = static_cast<float*>(workspace);
+    p.part_lse = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(rows * D * sizeof(float), 256));
+    if (static_cast<long long>(B) * Hkv > 2147483647ll) return SDPA_ERR_SHAPE;
+    dim3 grid(static_cast<unsigned>(B * Hkv), static_cast<unsigned>(n_splits), 1);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (padded_head_dim(D) == 128)
+        sdpa_fwd_kernel<128, true, true><<<grid, FwdCfg<128>::kThreads, FwdCfg<128>::kSmemBytes, s>>>(mq, mq, mq, p);
+    else
+        sdpa_fwd_kernel<64, true, true><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mq, mq, p);
+    SDPA_CUDA_TRY(cudaGetLastError());
+    sdpa_decode_combine_kernel<<<static_cast<unsigned>(B * Hq), 32, 0, s>>>(
+        p.part_o, p.part_lse, static_cast<__nv_bfloat16*>(o), lse, n_splits, B, Hq, D);
     SDPA_CUDA_TRY(cudaGetLastError());
     return SDPA_OK;
 }
