@@ -457,8 +457,15 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // thread 0 adds and passes the turn on two steps later, when `cp.async.bulk.wait_group 2` says that
         // the adds have been performed: their latency (L2 reduce throughput plus a round trip) is longer
         // than one step.  A wait that gives up raises the CTA's abort flag; the adds are then skipped.
-        int* pend_turn[2] = {nullptr, nullptr};  // thread 0: turns of the last two steps, oldest first
-        int pend_val[2] = {0, 0};
+        // turn counter of iteration i and this tile's rank on it (pure functions of i: nothing is carried
+        // from step to step in registers)
+        auto turn_of = [&](int i, int& rank) -> int* {
+            const int hh = g * G + i / per_head;
+            const int qq0 = step_of(i) * 64;
+            const int j_last = p.causal ? min(nt_seq - 1, (qq0 + 63 + off) >> 7) : nt_seq - 1;  // highest tile on the step
+            rank = j_last - jt;
+            return p.dq_turn + static_cast<size_t>(hh) * p.T + sp.gt0 + qq0;
+        };
         for (int it = 0; it < n_it && ok; ++it) {
             const int h = g * G + it / per_head;
             const int q0 = step_of(it) * 64;
@@ -475,22 +482,17 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tc_fence_before();
             mbar_arrive(&dq_empty[it & 1]);
             if (x == 0) SDPA_TR(4, it, 2);
-            int* turn = nullptr;
-            int rank = 0;
             if (det) {
-                const int j_last = p.causal ? min(nt_seq - 1, (q0 + 63 + off) >> 7) : nt_seq - 1;  // highest tile on this step
-                rank = j_last - jt;
-                turn = p.dq_turn + static_cast<size_t>(h) * p.T + sp.gt0 + q0;
-                if (x == 32) wait_turn(turn, rank, ctl, kBSiteTurn);  // sets the abort flag on failure
-                if (x == 0 && pend_turn[0] != nullptr) {
-                    bulk_wait<2>();  // all but the previous step's two groups: the adds of two steps ago are done
-                    SDPA_TR(4, it, 6);
-                    if (!*ctl.abort) release_turn(pend_turn[0], pend_val[0]);
-                    SDPA_TR(4, it, 7);
+                if (x == 32) {
+                    int rank;
+                    int* turn = turn_of(it, rank);
+                    wait_turn(turn, rank, ctl, kBSiteTurn);  // sets the abort flag on failure
                 }
-                if (x == 0) {
-                    pend_turn[0] = pend_turn[1]; pend_val[0] = pend_val[1];
-                    pend_turn[1] = turn;         pend_val[1] = rank + 1;
+                if (x == 0 && it >= 2) {
+                    bulk_wait<2>();  // all but the previous step's two groups: the adds of two steps ago are done
+                    int rank;
+                    int* turn = turn_of(it - 2, rank);
+                    if (!*ctl.abort) release_turn(turn, rank + 1);
                 }
             }
             // Two halves of 32 query rows, each its own bulk group: the rows of one half are rewritten
@@ -521,9 +523,12 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         if (x == 0) {
             bulk_wait<0>();
-            if (det && !*ctl.abort) {
-                if (pend_turn[0] != nullptr) release_turn(pend_turn[0], pend_val[0]);
-                if (pend_turn[1] != nullptr) release_turn(pend_turn[1], pend_val[1]);
+            if (det && ok && !*ctl.abort) {
+                for (int i = max(0, n_it - 2); i < n_it; ++i) {
+                    int rank;
+                    int* turn = turn_of(i, rank);
+                    release_turn(turn, rank + 1);
+                }
             }
         }
     } else if (warp == 13) {
