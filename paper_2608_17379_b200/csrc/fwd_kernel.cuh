@@ -43,8 +43,9 @@ struct FwdParams {
     int d;             // head dimension of the tensors (multiple of 8, <= D of the kernel; columns d..D-1 are zero padding)
     TensorLayout lay;  // strides of q / o (and of k / v for the non-paged kernel), lse
     // decode variant only: per key split, unnormalised-free partial results of every (sequence, head)
-    float* part_o;     // [n_splits, B, Hq, d] fp32: softmax-weighted average of V over the split's keys
-    float* part_lse;   // [n_splits, B, Hq] fp32: log-sum-exp over the split's keys (-inf for an empty split)
+    float* part_o;     // [2 * n_splits, B, Hq, d] fp32: softmax average of V over the keys of one slot of a split
+    float* part_lse;   // [2 * n_splits, B, Hq] fp32: log-sum-exp over those keys (-inf where there were none)
+    int tiles_per_split;  // decode variant: key tiles one CTA takes
     int head_chunk;    // (sequence, query head) pairs whose CTAs are launched interleaved
     float scale;       // softmax scale
     float scale_log2;  // scale * log2(e)
@@ -94,7 +95,8 @@ __global__ void __launch_bounds__(384, 1)
 sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
     using Cfg = FwdCfg<D>;
-    constexpr int S = Cfg::kStages;
+    // ring slots; the decode variant has no second Q tile and adds that buffer to the ring
+    constexpr int S = kDecode ? Cfg::kStages + 1 : Cfg::kStages;
 
     static_assert(!kDecode || kPaged, "the decode variant reads a paged cache");
     int b, h, g, r0, L, q_start;
@@ -160,13 +162,18 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int n_kv_all = (Lk + 127) >> 7;
     int tile_begin = 0;  // first key tile of this CTA (decode: the start of its split)
     if (kDecode) {
-        const int per_split = (n_kv_all + (int)gridDim.y - 1) / (int)gridDim.y;
+        const int per_split = p.tiles_per_split;  // key tiles per CTA, the same for every sequence
         tile_begin = (int)blockIdx.y * per_split;
-        n_kv[0] = min(n_kv_all, tile_begin + per_split) - tile_begin;
-        n_kv[1] = 0;
-        if (n_kv[0] <= 0) {  // nothing in this split: the combining kernel skips a partial whose lse is -inf
-            if ((int)threadIdx.x < G)
-                p.part_lse[(static_cast<size_t>(blockIdx.y) * p.B + b) * p.Hq + h + threadIdx.x] = -INFINITY;
+        const int n_mine = min(n_kv_all, tile_begin + per_split) - tile_begin;
+        // The two tile slots of the CTA work on the same query rows and take the split's key tiles in turn
+        // (slot t: tiles t, t+2, ...), each with its own running maximum, sum and accumulator, so that one
+        // slot's softmax overlaps the other's MMAs; they leave two partial results for the combining kernel.
+        n_kv[0] = max(0, (n_mine + 1) >> 1);
+        n_kv[1] = max(0, n_mine >> 1);
+        if (n_mine <= 0) {  // nothing in this split: the combining kernel skips a partial whose lse is -inf
+            if ((int)threadIdx.x < 2 * G)
+                p.part_lse[(static_cast<size_t>(2 * blockIdx.y + threadIdx.x / G) * p.B + b) * p.Hq + h + threadIdx.x % G] =
+                    -INFINITY;
             return;
         }
     } else {
@@ -174,12 +181,12 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         n_kv[0] = p.causal ? min(n_kv_all, ((q_start + 127 + off) >> 7) + 1) : n_kv_all;
         n_kv[1] = has1 ? (p.causal ? min(n_kv_all, ((q_start + 255 + off) >> 7) + 1) : n_kv_all) : 0;
     }
-    const int n_iter = max(n_kv[0], n_kv[1]);
+    const int n_iter = kDecode ? n_kv[0] + n_kv[1] : max(n_kv[0], n_kv[1]);  // decode: key tiles of the CTA
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;
-    uint8_t* sRing = smem + Cfg::kSmemQ;
+    uint8_t* sRing = kDecode ? sQ + Cfg::kTileBytes : smem + Cfg::kSmemQ;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kSmemQ + Cfg::kSmemRing);
     uint64_t* q_full = bars;               // [2]
     uint64_t* kv_full = bars + 2;          // [S]
@@ -201,8 +208,10 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int i = 0; i < 2; ++i) {
             mbar_init(&q_full[i], 1);
             mbar_init(&s_full[i], 1);
-            mbar_init(&p_full[i], 128);
-            mbar_init(&p_half[i], 128);
+            // decode: only the warps that own query heads (rows below G) take part in the softmax hand-shake
+            const int p_count = kDecode ? 32 * ((G + 31) / 32) : 128;
+            mbar_init(&p_full[i], p_count);
+            mbar_init(&p_half[i], p_count);
             mbar_init(&o_full[i], 1);
         }
         for (int i = 0; i < S; ++i) {
@@ -226,6 +235,95 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    // ------------------------------------------------------------ gathering producers (paged variants)
+    // Warps 9-11; in the decode variant also the softmax warps that own no query head.
+    // A gatherer's next item is n_gather items ahead; with more gatherers than ring slots it could run two
+    // revolutions of the ring ahead of the consumer, which the one-bit phase of an mbarrier cannot tell from
+    // one revolution (seen as a corrupted ring and a wait that ran out).  So at most S warps gather.
+    const int n_live = kDecode ? 2 * ((G + 31) / 32) : 8;  // softmax warps that do arithmetic
+    const int n_gather = min(3 + (8 - n_live), S);
+    auto gather_role = [&](int pw) {
+            // -------------------------------------------------------- gathering producers (warps 9-11, all lanes)
+            // K_j is ring item 2j, V_j item 2j+1; item `it` is gathered by gathering warp it % n_gather, so several
+            // tiles are in flight.  A tile's 128 rows come from the page-size-1 cache with 16-byte cp.async into the same
+            // 128B-swizzled layout a TMA load would produce; D/8 consecutive lanes copy one row (full lines in
+            // the cache), the page numbers travel by shuffle.  Rows past the sequence end and the padding
+            // columns are zero-filled (a masked P of exactly 0 must not meet garbage in V).
+            const int lane = tid & 31;
+            if (pw == 0 && lane == 0) {
+                // decode: the Q map's box is the G heads of the group for one token (G rows of the tile)
+                mbar_arrive_expect_tx(&q_full[0], kDecode ? static_cast<uint32_t>(G) * D * 2u : Cfg::kTileBytes);
+#pragma unroll
+                for (int a = 0; a < D / 64; ++a)
+                    SDPA_TMA_LOAD_ROWS(sQ + a * Cfg::kAtomBytes, &map_q, &q_full[0], a * 64, r0 + q_start, h, sp.bidx, p.lay.dense);
+                if (!kDecode && n_kv[1] > 0) {  // decode: both slots read the one Q tile
+                    mbar_arrive_expect_tx(&q_full[1], Cfg::kTileBytes);
+#pragma unroll
+                    for (int a = 0; a < D / 64; ++a)
+                        SDPA_TMA_LOAD_ROWS(sQ + Cfg::kTileBytes + a * Cfg::kAtomBytes, &map_q, &q_full[1], a * 64,
+                                    r0 + q_start + 128, h, sp.bidx, p.lay.dense);
+                }
+            }
+            constexpr int kLanesPerRow = D / 8;               // 16-byte chunks of a row
+            constexpr int kRowsPerCopy = 32 / kLanesPerRow;    // rows one warp-wide cp.async covers
+            const int my_c = lane % kLanesPerRow;
+            const int my_sub = lane / kLanesPerRow;
+            bool ok = true;
+            for (int it = pw; it < 2 * n_iter && ok; it += n_gather) {
+                // which tile ring item `it` is: K_0 V_0 K_1 V_1 ... in general; the decode variant consumes
+                // K_0 K_1 V_0 K_2 V_1 K_3 ... V_(n-2) V_(n-1) (two slots, each one tile ahead with its S)
+                int j = it >> 1, kv = it & 1;
+                if (kDecode) {
+                    if (it == 0) { j = 0; kv = 0; }
+                    else if (it == 1 && n_iter > 1) { j = 1; kv = 0; }
+                    else if (it <= 2 * n_iter - 3) { kv = (it & 1) ^ 1; j = kv ? (it - 2) >> 1 : (it + 1) >> 1; }
+                    else { kv = 1; j = it - n_iter; }
+                }
+                // cache row addresses of the rows lane, lane+32, lane+64, lane+96 of key tile j (0: past the end)
+                const __nv_bfloat16* cache = kv == 0 ? p.k_cache : p.v_cache;
+                unsigned long long row_ptr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int key = (tile_begin + j) * 128 + lane + 32 * i;
+                    unsigned long long ptr = 0ull;
+                    if (key < Lk) {
+                        const int pg = p.kv_indices[kbase + key];
+                        if (pg < 0 || pg >= p.num_pages)  // never read outside the cache
+                            atomicCAS(p.status, 0, kStatusBadCuSeqlens);
+                        else
+                            ptr = reinterpret_cast<unsigned long long>(cache + (static_cast<size_t>(pg) * p.Hkv + g) * p.d);
+                    }
+                    row_ptr[i] = ptr;
+                }
+                const int st = it % S;
+                ok = mbar_wait_warp(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
+                if (!ok) break;
+                // Per copy only the row address (two shuffles) and a constant XOR change: the lane's column
+                // chunk, its sub-row and the swizzle term they give are fixed.  row & 7 = (rr & 7) | my_sub
+                // because rr is a multiple of the rows per copy, so chunk ^ (row & 7) = (chunk ^ my_sub) ^ (rr & 7).
+                const bool col_real = my_c * 8 < p.d;
+                const uint32_t dst_lane = smem_u32(sRing + st * Cfg::kTileBytes) + (my_c >> 3) * Cfg::kAtomBytes + my_sub * 128;
+                const uint32_t swz_lane = static_cast<uint32_t>((my_c & 7) ^ my_sub);
+                const unsigned long long col_off = static_cast<unsigned long long>(my_c) * 16ull;
+#pragma unroll
+                for (int rr = 0; rr < 128; rr += kRowsPerCopy) {
+                    const unsigned long long base = __shfl_sync(0xffffffffu, row_ptr[rr >> 5], (rr + my_sub) & 31);
+                    const bool real = base != 0ull && col_real;
+                    const uint32_t dst = dst_lane + rr * 128 + ((swz_lane ^ (rr & 7)) << 4);
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst),
+                                 "l"(real ? base + col_off : reinterpret_cast<unsigned long long>(cache)), "r"(real ? 16u : 0u)
+                                 : "memory");
+                }
+                cp_async_commit();
+                // The item is handed over before this warp asks for its next slot: that slot is freed by MMAs
+                // which may themselves be waiting for this item.  The overlap comes from the other two warps.
+                cp_async_wait<0>();          // the copies have landed
+                fence_proxy_async_smem();    // make them visible to the tensor core's reads
+                mbar_arrive(&kv_full[st]);
+            }
+            cp_async_wait<0>();
+    };
+
     if (warp < 8) {
         // ------------------------------------------------------------ softmax groups
         setmaxnreg_inc<208>();
@@ -242,18 +340,19 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         float m = -INFINITY, l = 0.f;
         const int n = n_kv[t];
         bool ok = true;
+        if (kPaged && !warp_live) {
+            // decode: this warp owns no query head; it gathers K/V tiles instead (gatherers 3, 4, ...)
+            const int live_per_group = (G + 31) / 32;
+            const int pw = 3 + t * (4 - live_per_group) + ((warp & 3) - live_per_group);
+            if (pw < n_gather) gather_role(pw);
+            ok = false;  // nothing to store
+        }
         for (int j = 0; j < n && ok; ++j) {
             if (row_in_tile == 0) SDPA_TR(t, j, 0);
             ok = mbar_wait_warp(&s_full[t], j & 1, ctl, kSiteSFull);
             if (!ok) break;
             if (row_in_tile == 0) SDPA_TR(t, j, 1);
             tc_fence_after();
-            if (!warp_live) {
-                tc_fence_before();
-                mbar_arrive(&p_half[t]);
-                mbar_arrive(&p_full[t]);
-                continue;
-            }
             float s[128];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -268,7 +367,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                 for (int c = 0; c < 128; ++c) s[c] = 0.f;
             }
-            const int key0 = (tile_begin + j) * 128;
+            const int key0 = (tile_begin + (kDecode ? 2 * j + t : j)) * 128;
             const bool diag = p.causal && (key0 + 127 > q_start + t * 128 + off);
             if (diag || key0 + 128 > Lk) {
                 const int lim = p.causal ? min(row + off, Lk - 1) : (Lk - 1);  // last allowed key
@@ -356,10 +455,11 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (ok && n > 0) ok = mbar_wait_warp(&o_full[t], 0, ctl, kSiteOFull);
         if (kDecode) {
             // the G rows of the group leave as fp32 partial results of this key split
+            const size_t slot = (static_cast<size_t>(2 * blockIdx.y + t) * p.B + b) * p.Hq + h + row_in_tile;
+            if (n == 0 && valid) p.part_lse[slot] = -INFINITY;  // this slot had no key tile
             if (ok && n > 0 && warp_live) {
                 tc_fence_after();
                 const float inv_l = 1.0f / l;
-                const size_t slot = (static_cast<size_t>(blockIdx.y) * p.B + b) * p.Hq + h + row_in_tile;
                 float* dst = p.part_o + slot * p.d;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
@@ -426,72 +526,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     } else {
         setmaxnreg_dec<80>();
         if (warp >= 9 && kPaged) {
-            // -------------------------------------------------------- gathering producers (warps 9-11, all lanes)
-            // K_j is ring item 2j, V_j item 2j+1; item `it` is gathered by warp 9 + it % 3, so three tiles are
-            // in flight.  A tile's 128 rows come from the page-size-1 cache with 16-byte cp.async into the same
-            // 128B-swizzled layout a TMA load would produce; D/8 consecutive lanes copy one row (full lines in
-            // the cache), the page numbers travel by shuffle.  Rows past the sequence end and the padding
-            // columns are zero-filled (a masked P of exactly 0 must not meet garbage in V).
-            const int lane = tid & 31;
-            const int pw = warp - 9;
-            if (pw == 0 && lane == 0) {
-                // decode: the Q map's box is the G heads of the group for one token (G rows of the tile)
-                mbar_arrive_expect_tx(&q_full[0], kDecode ? static_cast<uint32_t>(G) * D * 2u : Cfg::kTileBytes);
-#pragma unroll
-                for (int a = 0; a < D / 64; ++a)
-                    SDPA_TMA_LOAD_ROWS(sQ + a * Cfg::kAtomBytes, &map_q, &q_full[0], a * 64, r0 + q_start, h, sp.bidx, p.lay.dense);
-                if (n_kv[1] > 0) {
-                    mbar_arrive_expect_tx(&q_full[1], Cfg::kTileBytes);
-#pragma unroll
-                    for (int a = 0; a < D / 64; ++a)
-                        SDPA_TMA_LOAD_ROWS(sQ + Cfg::kTileBytes + a * Cfg::kAtomBytes, &map_q, &q_full[1], a * 64,
-                                    r0 + q_start + 128, h, sp.bidx, p.lay.dense);
-                }
-            }
-            constexpr int kLanesPerRow = D / 8;               // 16-byte chunks of a row
-            constexpr int kRowsPerCopy = 32 / kLanesPerRow;    // rows one warp-wide cp.async covers
-            const int my_c = lane % kLanesPerRow;
-            const int my_sub = lane / kLanesPerRow;
-            bool ok = true;
-            for (int it = pw; it < 2 * n_iter && ok; it += 3) {
-                const int j = it >> 1, kv = it & 1;
-                int page[4];  // pages of the rows lane, lane+32, lane+64, lane+96 of key tile j (-1: past the end)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int key = (tile_begin + j) * 128 + lane + 32 * i;
-                    int pg = -1;
-                    if (key < Lk) {
-                        pg = p.kv_indices[kbase + key];
-                        if (pg < 0 || pg >= p.num_pages) {  // never read outside the cache
-                            atomicCAS(p.status, 0, kStatusBadCuSeqlens);
-                            pg = -1;
-                        }
-                    }
-                    page[i] = pg;
-                }
-                const int st = it % S;
-                ok = mbar_wait_warp(&kv_empty[st], ((it / S) & 1) ^ 1, ctl, kSiteKvEmpty);
-                if (!ok) break;
-                uint8_t* dst = sRing + st * Cfg::kTileBytes;
-                const __nv_bfloat16* cache = kv == 0 ? p.k_cache : p.v_cache;
-                const bool col_real = my_c * 8 < p.d;
-#pragma unroll
-                for (int rr = 0; rr < 128; rr += kRowsPerCopy) {
-                    const int row = rr + my_sub;
-                    const int pg = __shfl_sync(0xffffffffu, page[rr >> 5], row & 31);  // rr / 32 == row / 32
-                    const bool real = pg >= 0 && col_real;
-                    const __nv_bfloat16* src = cache + (static_cast<size_t>(pg >= 0 ? pg : 0) * p.Hkv + g) * p.d;
-                    cp_async_16(dst + (my_c >> 3) * Cfg::kAtomBytes + sw128_offset(row, my_c & 7), real ? src + my_c * 8 : src,
-                                real ? 16u : 0u);
-                }
-                cp_async_commit();
-                // The item is handed over before this warp asks for its next slot: that slot is freed by MMAs
-                // which may themselves be waiting for this item.  The overlap comes from the other two warps.
-                cp_async_wait<0>();          // the copies have landed
-                fence_proxy_async_smem();    // make them visible to the tensor core's reads
-                mbar_arrive(&kv_full[st]);
-            }
-            cp_async_wait<0>();
+            gather_role(warp - 9);
         } else if (warp == 9) {
             // -------------------------------------------------------- TMA producer
             if (elect_one()) {
@@ -558,6 +593,63 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 };
                 bool ok = true;
                 int it = 0;  // ring consumer counter: K_j is item 2j, V_j is item 2j+1
+                if (kDecode) {
+                    // two slots on the same query rows (both use Q tile 0), slot t takes key tiles t, t+2, ...
+                    const int n = n_iter;
+                    auto next_item = [&]() {
+                        const int st = it % S;
+                        const bool w = mbar_wait(&kv_full[st], (it / S) & 1, ctl, kSiteKvFull);
+                        ++it;
+                        if (w) tc_fence_after();
+                        ok = w;
+                        return st;
+                    };
+                    auto issue_qk0 = [&](int t, int st) {
+                        const uint64_t b0 = k_desc + static_cast<uint64_t>(st * (Cfg::kTileBytes >> 4));
+                        const uint32_t d = tmem + t * 128;
+#pragma unroll
+                        for (int kk = 0; kk < Cfg::kKSteps; ++kk) {
+                            const uint64_t off = static_cast<uint64_t>(((kk >> 2) * Cfg::kAtomBytes + (kk & 3) * 32) >> 4);
+                            umma_ss(d, q_desc0 + off, b0 + off, idesc_qk, kk > 0);
+                        }
+                    };
+                    ok = mbar_wait(&q_full[0], 0, ctl, kSiteQFull);
+                    for (int t = 0; t < 2 && t < n && ok; ++t) {
+                        const int st = next_item();
+                        if (!ok) break;
+                        issue_qk0(t, st);
+                        umma_commit(&s_full[t]);
+                        umma_commit(&kv_empty[st]);
+                    }
+                    for (int j = 0; j < n && ok; ++j) {
+                        const int t = j & 1, i = j >> 1;
+                        const int st_v = next_item();
+                        if (!ok) break;
+                        ok = mbar_wait(&p_half[t], i & 1, ctl, kSitePFull);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(t, st_v, i > 0, 0);
+                        ok = mbar_wait(&p_full[t], i & 1, ctl, kSitePFull);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(t, st_v, i > 0, 1);
+                        umma_commit(&kv_empty[st_v]);
+                        if (j + 2 < n) {
+                            const int st_k = next_item();
+                            if (!ok) break;
+                            issue_qk0(t, st_k);
+                            umma_commit(&s_full[t]);
+                            umma_commit(&kv_empty[st_k]);
+                        } else {
+                            umma_commit(&o_full[t]);
+                        }
+                    }
+                    if (!ok) {
+                        umma_commit(drain);
+                        mbar_wait(drain, 0, ctl, kSiteDrain);
+                    }
+                    goto mma_done;
+                }
                 ok = mbar_wait(&q_full[0], 0, ctl, kSiteQFull);
                 if (ok) ok = mbar_wait(&kv_full[0], 0, ctl, kSiteKvFull);
                 if (ok) {
@@ -622,6 +714,7 @@ sdpa_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     umma_commit(drain);
                     mbar_wait(drain, 0, ctl, kSiteDrain);
                 }
+            mma_done:;
             }
         }
     }

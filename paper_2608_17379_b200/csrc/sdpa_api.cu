@@ -350,18 +350,24 @@ extern "C" int sdpa_fwd_paged(const void* q, const void* k_cache, const void* v_
     return SDPA_OK;
 }
 
-// Key splits of the decode path: about two CTAs per SM of a B200 over all (sequence, kv head) pairs, at most
-// one split per 128-key tile of the longest sequence.
+// Decode path: key tiles per CTA and the number of key splits that follows for the longest sequence.  Every
+// CTA takes the same number of tiles, so short sequences use fewer CTAs (their surplus splits leave at once).
+// A CTA costs about 5 us before its first tile is done, so CTAs are kept long: at least 8 tiles, and enough
+// that all (sequence, kv head) groups at full length would fit one wave of a B200's 148 SMs.
+static int decode_tiles_per_split(int B, int Hkv, int max_seqlen_k) {
+    const long long tiles = std::max(1, (max_seqlen_k + 127) / 128);
+    const long long one_wave = (tiles * B * Hkv + 147) / 148;
+    return static_cast<int>(std::max<long long>(1, std::min<long long>(std::max<long long>(8, one_wave), tiles)));
+}
 static int decode_splits(int B, int Hkv, int max_seqlen_k) {
-    const long long groups = static_cast<long long>(B) * Hkv;
     const int tiles = std::max(1, (max_seqlen_k + 127) / 128);
-    const long long want = (2 * 148 + groups - 1) / groups;
-    return static_cast<int>(std::max<long long>(1, std::min<long long>(want, tiles)));
+    const int tps = decode_tiles_per_split(B, Hkv, max_seqlen_k);
+    return (tiles + tps - 1) / tps;
 }
 
 extern "C" size_t sdpa_decode_paged_workspace_bytes(int B, int Hq, int Hkv, int D, int max_seqlen_k) {
     if (B < 1 || Hq < 1 || Hkv < 1 || max_seqlen_k < 0 || D < 8 || D > 128 || (D % 8) != 0 || Hq % Hkv != 0) return 0;
-    const size_t rows = static_cast<size_t>(decode_splits(B, Hkv, max_seqlen_k)) * B * Hq;
+    const size_t rows = static_cast<size_t>(2 * decode_splits(B, Hkv, max_seqlen_k)) * B * Hq;  // two slots per split
     return align_up(rows * D * sizeof(float), 256) + align_up(rows * sizeof(float), 256);
 }
 
@@ -406,7 +412,8 @@ extern "C" int sdpa_decode_paged(const void* q, const void* k_cache, const void*
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.head_chunk = 1;
-    const size_t rows = static_cast<size_t>(n_splits) * B * Hq;
+    p.tiles_per_split = decode_tiles_per_split(B, Hkv, max_seqlen_k);
+    const size_t rows = static_cast<size_t>(2 * n_splits) * B * Hq;  // every CTA leaves two partial results
     p.part_o = static_cast<float*>(workspace);
     p.part_lse = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(rows * D * sizeof(float), 256));
     if (static_cast<long long>(B) * Hkv > 2147483647ll) return SDPA_ERR_SHAPE;
@@ -418,7 +425,7 @@ extern "C" int sdpa_decode_paged(const void* q, const void* k_cache, const void*
         sdpa_fwd_kernel<64, true, true><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, s>>>(mq, mq, mq, p);
     SDPA_CUDA_TRY(cudaGetLastError());
     sdpa_decode_combine_kernel<<<static_cast<unsigned>(B * Hq), 32, 0, s>>>(
-        p.part_o, p.part_lse, static_cast<__nv_bfloat16*>(o), lse, n_splits, B, Hq, D);
+        p.part_o, p.part_lse, static_cast<__nv_bfloat16*>(o), lse, 2 * n_splits, B, Hq, D);
     SDPA_CUDA_TRY(cudaGetLastError());
     return SDPA_OK;
 }
