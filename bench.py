@@ -176,6 +176,98 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_decode(args):
+    """Secondary workload (not the default bench line): paged GQA decode, one query token per sequence
+    over a page-size-1 KV cache (the paper's decode operator at a size that fills the GPU: batch 64,
+    4096 keys per sequence, 32 query / 8 kv heads, D = 128, pages drawn at random from the cache).
+    One step = one sdpa_decode_paged call (two kernels); the metric is K/V bytes read per second, the
+    quantity this path is bound by."""
+    B, Lk, Hq, Hkv, D = 64, 4096, 32, 8, 128
+    num_pages = B * Lk + 1000
+    kv_bytes = B * Lk * Hkv * D * 2 * 2
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return
+        from oracle import paged as PG
+        rng = np.random.default_rng(3)
+        nb = 2  # sequences per step of the sample
+        secs = []
+        q = rng.standard_normal((nb, Hq, D)); kc = rng.standard_normal((nb * Lk, Hkv, D)); vc = rng.standard_normal((nb * Lk, Hkv, D))
+        cu = np.arange(nb + 1, dtype=np.int32); ip = (np.arange(nb + 1) * Lk).astype(np.int32)
+        idx = rng.permutation(nb * Lk).astype(np.int32)
+        for i in range(args.warmup + args.steps):
+            t0 = time.perf_counter()
+            PG.sdpa_fwd_paged(q, kc, vc, cu, ip, idx, True, D ** -0.5)
+            if i >= args.warmup:
+                secs.append(time.perf_counter() - t0)
+        value = nb * Lk * Hkv * D * 2 * 2 * len(secs) / sum(secs) / 1e9
+        print(json.dumps({"impl": "reference", "metric": "paged decode K/V GB/s", "value": value, "unit": "GB/s",
+                          "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": {"workload": "paged decode", "note": f"fp64 numpy oracle, {nb} of {B} sequences per step"},
+                          "cpu_baseline": {"value": value, "unit": "GB/s", "cores": os.cpu_count(), "kind": "oracle",
+                                           "sample": f"{nb} of {B} sequences per step"},
+                          "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}), flush=True)
+        return
+    from paper_2608_17379_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    g = torch.Generator(device="cuda"); g.manual_seed(11)
+    q = torch.randn(B, Hq, D, device="cuda", generator=g).bfloat16()
+    kc = torch.randn(num_pages, Hkv, D, device="cuda", generator=g).bfloat16()
+    vc = torch.randn(num_pages, Hkv, D, device="cuda", generator=g).bfloat16()
+    ip = torch.arange(B + 1, dtype=torch.int32, device="cuda") * Lk
+    idx = torch.randperm(num_pages, device="cuda", generator=g)[:B * Lk].int()
+    ws = torch.empty(binding.load().sdpa_decode_paged_workspace_bytes(B, Hq, Hkv, D, Lk), dtype=torch.uint8, device="cuda")
+    o = torch.empty_like(q); lse = torch.empty(Hq, B, device="cuda")
+    q_h = q.cpu().pin_memory(); o_h = torch.empty_like(q_h).pin_memory()
+    step = lambda: binding.sdpa_decode_paged(q, kc, vc, ip, idx, Lk, D ** -0.5, o=o, lse=lse, workspace=ws)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    K_ = args.steps
+    with ClockSampler(0) as clocks:
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(K_):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / K_
+    s0, s1 = ev(), ev()
+    s0.record()
+    for _ in range(3):  # end to end: the query comes from the host and the result goes back; the cache lives on the GPU
+        q.copy_(q_h, non_blocking=True)
+        step()
+        o_h.copy_(o, non_blocking=True)
+    s1.record()
+    torch.cuda.synchronize()
+    e2e_ms = s0.elapsed_time(s1) / 3
+    assert binding.query_status() == (0, 0)
+    peaks = measured_peaks()
+    gbs = kv_bytes / (ms * 1e-3) / 1e9
+    line = {"metric": "paged decode K/V GB/s (bf16, device-timed)", "value": gbs, "unit": "GB/s", "n_gpus": 1,
+            "steps": K_, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"paged decode B={B} Lk={Lk} Hq={Hq} Hkv={Hkv} D={D} page size 1",
+                       "l2": f"K/V pages read per step = {kv_bytes / 1e6:.0f} MB exceed the 126 MB L2; no flush"},
+            "roofline": {"bound": "hbm", "kernel": "sdpa_fwd_kernel<128,true,true>", "achieved": gbs,
+                         "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]),
+                         "peak_source": f"{peaks['_source']} copy bandwidth",
+                         # dram read + write of one launch of the main kernel, from one ncu capture of this
+                         # command (summary kept under profiles/)
+                         "traffic": 1075622912 + 6904064, "traffic_unit": "bytes per launch (ncu dram read+write)",
+                         "algorithmic_bytes_per_launch": kv_bytes},
+            "e2e": {"value": kv_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": q.numel() * 2, "d2h_bytes_per_step": q.numel() * 2},
+            "gpu_launches": 2 * K_, "clocks": clocks.summary()}
+    print(json.dumps(line), flush=True)
+
+
 def run_gemm(args):
     """Secondary workload (not the default bench line): the paper's bf16 GEMM C = A B^T,
     A 8192x5120, B 7168x5120, seeded synthetic N(0,1) inputs.  One step = one GEMM."""
@@ -261,10 +353,13 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c3", choices=list(W.CONFIG_NAMES) + ["gemm"])
+    ap.add_argument("--config", default="c3", choices=list(W.CONFIG_NAMES) + ["gemm", "decode"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.config == "decode":
+        run_decode(args)
+        return
     if args.config == "gemm":
         run_gemm(args)
         return
