@@ -336,13 +336,14 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int i = i4 * 4 + e;
-                        float v = fast_exp2(fmaf(__uint_as_float(sr[i]), p.scale_log2, -lv[e]));
-                        if (need_mask) {
-                            const int qq = q0 + c * 32 + i;
-                            if (!key_ok || (p.causal && key > qq + off)) v = 0.f;
-                        }
-                        pr[c * 32 + i] = v;
+                        pr[c * 32 + i] = fast_exp2(fmaf(__uint_as_float(sr[i]), p.scale_log2, -lv[e]));
                     }
+                }
+                if (need_mask) {  // diagonal and tail steps only: kept out of the common path
+                    const int q_lim = key - off;  // under a causal mask this key is seen by queries >= q_lim
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (!key_ok || (p.causal && q0 + c * 32 + i < q_lim)) pr[c * 32 + i] = 0.f;
                 }
                 uint32_t pk[16];
 #pragma unroll
