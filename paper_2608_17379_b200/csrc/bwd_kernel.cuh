@@ -324,11 +324,13 @@ sdpa_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (r == 0) SDPA_TR(0, s, 1);
             tc_fence_after();
             float pr[64];
+            uint32_t sr_all[2][32];  // both halves of the step's scores are requested before the first wait
+            tmem_ld_x32(tS, sr_all[0]);
+            tmem_ld_x32(tS + 32, sr_all[1]);
+            tmem_wait_ld();
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
-                uint32_t sr[32];
-                tmem_ld_x32(tS + c * 32, sr);
-                tmem_wait_ld();
+                const uint32_t (&sr)[32] = sr_all[c];
 #pragma unroll
                 for (int i4 = 0; i4 < 8; ++i4) {
                     const float4 l4 = lse4[c * 8 + i4];
