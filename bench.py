@@ -32,9 +32,9 @@ METRIC = "SDPA fwd+bwd TFLOPS (bf16, device-timed)"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this same command on
 # the c3 workload (its summary is kept under profiles/); null for other workloads.
-NCU_DRAM_TRAFFIC_C3 = {"sdpa_bwd_kernel<128>": 365212928 + 155866112, "sdpa_fwd_kernel<128>": 101782784 + 36194304}
+NCU_DRAM_TRAFFIC_C3 = {"sdpa_bwd_kernel<128>": 371038720 + 158737920, "sdpa_fwd_kernel<128>": 101588992 + 35575296}
 # sm__pipe_tensor_cycles_active.avg.pct_of_peak_sustained_active of the same capture (clock independent)
-NCU_TENSOR_ACTIVE_PCT_C3 = {"sdpa_bwd_kernel<128>": 57.76, "sdpa_fwd_kernel<128>": 58.01}
+NCU_TENSOR_ACTIVE_PCT_C3 = {"sdpa_bwd_kernel<128>": 58.54, "sdpa_fwd_kernel<128>": 56.51}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
