@@ -133,7 +133,10 @@ sdpa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloa
 __global__ void __launch_bounds__(256)
 sdpa_bwd_dq_convert_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq, long long n8, float scale,
                            int T, int Hq, int D, int d, const TensorLayout lay) {
-    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;  // output group of 8
+    // Blocks walk the tokens from the last one down: the rows the main kernel reduced into most recently are
+    // still in the L2, the first ones are not; reading the hot rows first keeps them from being evicted by
+    // this kernel's own traffic.
+    const long long i = (static_cast<long long>(gridDim.x) - 1 - blockIdx.x) * blockDim.x + threadIdx.x;  // output group of 8
     if (i >= n8) return;
     const int d8 = d / 8;  // output rows have d columns, accumulator rows D (padded)
     const int part = static_cast<int>(i % d8);
