@@ -1,10 +1,12 @@
 /*
  * sdpa.h - C ABI of the B200 (sm_100a) bf16 scaled-dot-product-attention library.
  *
- * One forward and one backward entry point over packed (variable-length) batches with
- * grouped-query heads.  Every step of the path runs in this library's own CUDA kernels
- * (TMA-staged tiles, tcgen05 MMAs with TMEM accumulators); there is no CPU path and no call
- * into any attention/GEMM library.
+ * The primary pair is sdpa_fwd / sdpa_bwd over packed (variable-length) batches with grouped-query
+ * heads; the other entry points are the same two passes for other layouts and shapes (dense
+ * [B, H, S, D] tensors, separate key lengths, a paged KV cache, decode, a reproducible backward, host
+ * buffers, built-in scratch) and the paper's bf16 GEMM.  Every step of the path runs in this library's
+ * own CUDA kernels (TMA-staged tiles, tcgen05 MMAs with TMEM accumulators); there is no CPU path and
+ * no call into any attention/GEMM library.
  *
  * Conventions shared by all entry points
  * --------------------------------------
@@ -56,7 +58,7 @@ extern "C" {
 #define SDPA_ERR_STATIC_SCRATCH (-7) /* problem needs more than SDPA_STATIC_SCRATCH_BYTES of built-in scratch */
 
 #define SDPA_STATUS_TIMEOUT 1        /* a device-side wait gave up; outputs of that call are invalid */
-#define SDPA_STATUS_BAD_CU_SEQLENS 2 /* cu_seqlens contradicts total_tokens / max_seqlen */
+#define SDPA_STATUS_BAD_CU_SEQLENS 2 /* cu_seqlens / page table contradicts the sizes given, or breaks a length rule */
 #define SDPA_STATUS_INTERNAL 3       /* a kernel found its own launch preconditions violated */
 
 /*
